@@ -1,0 +1,170 @@
+/*
+ * libsmoothrot: the W4A4 SmoothRot linear layer on one NVIDIA B200 (sm_100a).
+ *
+ * The library implements the quantized linear layer that the SmoothRot method
+ * produces.  Notation (the paper's, with PyTorch's weight layout):
+ *
+ *   X  [M x K] fp16   activations, one row per token (K = input channels)
+ *   W  [N x K] fp16   weights, one row per output channel;  Y = X W^T
+ *   s  [K]     fp32   smoothing scales, Lambda = diag(s)
+ *   d  [K]     fp32   +1/-1 sign diagonal that randomises the Hadamard matrix
+ *   H          +1/-1  Hadamard matrix of order K (H H^T = K I):
+ *                     K = 2^p : Sylvester / Walsh, H[i][j] = (-1)^popcount(i & j)
+ *                     K = 28 * 2^p : kron(H28, H_{2^p}), index j = a * 2^p + b,
+ *                     H28 = Paley construction I over GF(27) (smoothrot_paley28)
+ *
+ * The equivalent transformation (Eq. 2 of the paper) is
+ *   Y = (X diag(pre_x) H / sqrt(K)) (W diag(pre_w) H / sqrt(K))^T,
+ *   pre_x = d / s,  pre_w = s * d,
+ * i.e. A = (H Lambda)^-1 of the Methodology section with the random signs
+ * merged into the diagonal.  Both factors are quantized to signed 4-bit codes
+ * (Eq. 1, symmetric form, codes in [-8, 7]) with one fp32 step size per row.
+ *
+ * Packed INT4 layout (used for Xq and Wq): row-major, K/2 bytes per row; byte
+ * i of a row holds code 2i in bits 0-3 and code 2i+1 in bits 4-7, each as
+ * 4-bit two's complement.
+ *
+ * Conventions for every call
+ *   - All tensor pointers are DEVICE pointers unless marked "host".  The
+ *     caller owns every buffer; the library allocates nothing and keeps no
+ *     reference after the work it enqueued has run.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls only enqueue work; they do not synchronise.
+ *   - Leading dimensions (ldx, ldw, ldy) count elements, not bytes.
+ *   - fp16 inputs must be 16-byte aligned with leading dimensions that are
+ *     multiples of 8; packed tensors must be 16-byte aligned.
+ *   - K must be 2^p with 7 <= p <= 13, or 28 * 2^p with 3 <= p <= 9.
+ *   - Return value: SMOOTHROT_OK (0) or a negative smoothrot_status.  On an
+ *     error nothing has been enqueued.  A size of zero rows is valid and
+ *     enqueues nothing.
+ */
+#ifndef SMOOTHROT_H_
+#define SMOOTHROT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SMOOTHROT_OK = 0,
+  SMOOTHROT_INVALID_ARG = -1,         /* null pointer, negative size, bad ratio */
+  SMOOTHROT_UNSUPPORTED_K = -2,       /* K is not one of the supported orders */
+  SMOOTHROT_BAD_ALIGNMENT = -3,       /* pointer or leading dimension misaligned */
+  SMOOTHROT_WORKSPACE_TOO_SMALL = -4, /* see smoothrot_workspace_bytes */
+  SMOOTHROT_CUDA_ERROR = -5,          /* a CUDA runtime / driver call failed */
+  SMOOTHROT_DEVICE_TIMEOUT = -6       /* a bounded wait inside a kernel ran out */
+} smoothrot_status;
+
+/* Host. Text for a status code; never NULL. */
+const char* smoothrot_status_string(int status);
+
+/*
+ * Scale calibration.  Methodology section:
+ *     s_j = max|X_j|^alpha / max|W_j|^(1 - alpha)
+ * with max|X_j| taken over all calibration tokens of the layer's raw input
+ * and max|W_j| over the output channels of the original weights.
+ *
+ * Call once per calibration batch.  Every call folds the batch into the
+ * running per-channel maximum  amax[j] = max(amax[j], max_t |X[t][j]|);
+ * the caller zero-fills amax before the first batch.  X may be NULL with
+ * T = 0.  When `finalize` is non-zero the call also reads W [N x K] and writes
+ *     s[j]     = max(amax[j], eps)^alpha / max(wmax[j], eps)^(1 - alpha),
+ *                floored at eps = 1e-5  (fp64 arithmetic, rounded to fp32)
+ * and, if `d` is non-NULL, the two diagonals the other calls take:
+ *     pre_w[j] = s[j] * d[j]          (for smoothrot_fuse_weights)
+ *     pre_x[j] = d[j] / s[j]          (for smoothrot_quant_act)
+ * pre_w_out / pre_x_out may each be NULL.  s_out doubles as the scratch for
+ * max|W_j| while the call runs.  W, s_out are ignored when finalize == 0.
+ */
+int smoothrot_calibrate(const void* X_f16, int64_t T, int64_t K, int64_t ldx,
+                        const void* W_f16, int64_t N, int64_t ldw,
+                        float alpha, int finalize,
+                        float* amax_inout, float* s_out,
+                        const float* d, float* pre_w_out, float* pre_x_out,
+                        void* stream);
+
+/*
+ * Offline weight path (Methodology section; Fig. 2's down-projection block
+ * "H Lambda W"; Experimental settings, "Quantization": per-channel symmetric
+ * round-to-nearest 4-bit weights).  For every row n of W:
+ *     w^   = (W[n][:] * pre) H / sqrt(K)            pre = s * d, or NULL = ones
+ *     dw[n]= clip_w * max|w^| / 7                   (1.0 if the row is all zero)
+ *     code = clamp(round_half_even(w^ / dw[n]), -8, 7),  packed 2 per byte
+ * Wq_out is [N x K/2] bytes, dw_out [N] fp32.  0 < clip_w <= 1.
+ */
+int smoothrot_fuse_weights(const void* W_f16, int64_t N, int64_t K, int64_t ldw,
+                           const float* pre, float clip_w,
+                           uint8_t* Wq_out, float* dw_out, void* stream);
+
+/*
+ * Online activation path (Fig. 2, "hadamard" then "quantize" before the
+ * down-projection; Experimental settings, "Quantization": per-token symmetric
+ * 4-bit activations with a constant clip ratio, 0.9 in the paper).  For every
+ * token m:
+ *     x^   = (X[m][:] * pre) H / sqrt(K)            pre = d / s, or NULL when
+ *                                                   Lambda^-1 already sits in
+ *                                                   the producing layer
+ *     dx[m]= clip_a * max|x^| / 7                   (1.0 if the row is all zero)
+ *     code = clamp(round_half_even(x^ / dx[m]), -8, 7),  packed 2 per byte
+ * Xq_out is [M x K/2] bytes, dx_out [M] fp32.  0 < clip_a <= 1.
+ */
+int smoothrot_quant_act(const void* X_f16, int64_t M, int64_t K, int64_t ldx,
+                        const float* pre, float clip_a,
+                        uint8_t* Xq_out, float* dx_out, void* stream);
+
+/*
+ * The quantized layer (Eq. 2's product on the integer codes of Eq. 1, then
+ * Eq. 1's dequantizer Q(x) = x_int * step applied to both factors):
+ *     acc[m][n] = sum_k Xq[m][k] * Wq[n][k]                    (int32, exact)
+ *     Y[m][n]   = fp16( float(acc[m][n]) * dx[m] * dw[n] )
+ * Xq [M x K/2], Wq [N x K/2] packed; dx [M], dw [N] fp32; Y [M x ldy] fp16
+ * with ldy >= N, ldy a multiple of 8, Y 16-byte aligned.  K must be a multiple
+ * of 128 and at most 65536; any M >= 0 and any N >= 0 that is a multiple of 8.
+ * `workspace` must hold smoothrot_workspace_bytes(M, N, K) bytes (it may be
+ * NULL when that is 0); its contents on entry do not matter.
+ */
+int smoothrot_linear(const uint8_t* Xq, const float* dx, int64_t M,
+                     const uint8_t* Wq, const float* dw, int64_t N, int64_t K,
+                     void* Y_f16, int64_t ldy,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
+/* Host. Scratch bytes smoothrot_linear / smoothrot_debug_gemm_i32 need for
+ * this shape (0 for shapes that need none). */
+size_t smoothrot_workspace_bytes(int64_t M, int64_t N, int64_t K);
+
+/*
+ * Test exports: values the fused kernels never write to memory.
+ *   smoothrot_debug_hadamard: Y[m][:] = (X[m][:] * pre) H / sqrt(K) as fp32
+ *     [M x K], the rotation alone (Methodology section).
+ *   smoothrot_debug_gemm_i32: the int32 accumulators acc [M x N] of
+ *     smoothrot_linear, computed by the same tensor-core kernel.
+ */
+int smoothrot_debug_hadamard(const void* X_f16, int64_t M, int64_t K, int64_t ldx,
+                             const float* pre, float* Y_f32, void* stream);
+int smoothrot_debug_gemm_i32(const uint8_t* Xq, int64_t M, const uint8_t* Wq, int64_t N,
+                             int64_t K, int32_t* acc,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/* Host. Writes the library's own order-28 Paley matrix, row-major, entries
+ * +1 / -1, into out[784] (a host buffer). */
+int smoothrot_paley28(int8_t* out_host);
+
+/*
+ * Host, synchronous.  Kernels never spin without bound: a wait that runs out
+ * records a non-zero code in a device-side status word and the kernel
+ * returns.  This call copies that word for the current device into
+ * *status_host (0 = no timeout so far) and clears it when `clear` is non-zero.
+ */
+int smoothrot_device_status(int* status_host, int clear);
+
+/* Host. Number of kernels this library has launched since it was loaded
+ * (all devices, all streams); used by the benchmark's launch count. */
+int64_t smoothrot_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SMOOTHROT_H_ */

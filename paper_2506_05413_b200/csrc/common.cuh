@@ -1,0 +1,51 @@
+// Shared host-side helpers of libsmoothrot (argument checks, launch counting).
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+
+#include "smoothrot.h"
+
+namespace smoothrot {
+
+// Number of kernels launched by the library (reported by smoothrot_launch_count).
+extern std::atomic<int64_t> g_launches;
+
+inline void count_launch(int n = 1) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline bool is_pow2(int64_t v) { return v > 0 && (v & (v - 1)) == 0; }
+
+inline int ilog2(int64_t v) {
+  int l = 0;
+  while ((int64_t(1) << l) < v) ++l;
+  return l;
+}
+
+// K = base * n with base 1 (Walsh, n = 2^p, 7 <= p <= 13) or base 28
+// (Paley x Walsh, n = 2^p, 3 <= p <= 9).  Returns false if K is neither.
+inline bool split_order(int64_t K, int* base, int* n, int* logn) {
+  if (is_pow2(K)) {
+    int l = ilog2(K);
+    if (l < 7 || l > 13) return false;
+    *base = 1; *n = int(K); *logn = l;
+    return true;
+  }
+  if (K > 0 && K % 28 == 0 && is_pow2(K / 28)) {
+    int l = ilog2(K / 28);
+    if (l < 3 || l > 9) return false;
+    *base = 28; *n = int(K / 28); *logn = l;
+    return true;
+  }
+  return false;
+}
+
+inline int launch_status() {
+  return cudaGetLastError() == cudaSuccess ? SMOOTHROT_OK : SMOOTHROT_CUDA_ERROR;
+}
+
+}  // namespace smoothrot

@@ -1,0 +1,450 @@
+// Row transform kernels of libsmoothrot:  v = (x * pre) H / sqrt(K)  followed by
+// per-row symmetric 4-bit quantization and packing (two codes per byte).
+//
+// Serves three entry points: smoothrot_quant_act (online activation path),
+// smoothrot_fuse_weights (offline weight path, same map with another diagonal
+// and clip ratio) and smoothrot_debug_hadamard (the rotation alone, fp32 out).
+//
+// Kernels
+//   rotate_generic_kernel   any supported K; one CTA per row, the row lives in
+//                           shared memory as fp32, butterflies three bits at a
+//                           time, the order-28 factor by a table product.
+//   walsh4096_kernel        K = 4096: 64 threads per row, 64 values per thread,
+//                           6 + 6 butterfly stages in registers around one
+//                           shared-memory transpose, codes assembled with warp
+//                           shuffles so that every global access is coalesced.
+//   paley512_kernel         K = 14336 = 28 x 512: see below.
+#include "common.cuh"
+
+namespace smoothrot {
+
+// ---------------------------------------------------------------------------
+// Order-28 Hadamard matrix, Paley construction I over GF(27).
+// GF(27) = GF(3)[x]/(x^3 + 2x + 1); element (c0, c1, c2) has index c0 + 3 c1 + 9 c2.
+// ---------------------------------------------------------------------------
+struct Gf27 {
+  int c0, c1, c2;
+};
+
+__host__ __device__ constexpr Gf27 gf_from_index(int e) { return Gf27{e % 3, (e / 3) % 3, e / 9}; }
+__host__ __device__ constexpr int gf_to_index(Gf27 v) { return v.c0 + 3 * v.c1 + 9 * v.c2; }
+
+__host__ __device__ constexpr Gf27 gf_diff(Gf27 a, Gf27 b) {
+  return Gf27{(a.c0 - b.c0 + 3) % 3, (a.c1 - b.c1 + 3) % 3, (a.c2 - b.c2 + 3) % 3};
+}
+
+// Product modulo x^3 + 2x + 1:  x^3 = x + 2 and x^4 = x^2 + 2x over GF(3).
+__host__ __device__ constexpr Gf27 gf_prod(Gf27 a, Gf27 b) {
+  int p0 = a.c0 * b.c0;
+  int p1 = a.c0 * b.c1 + a.c1 * b.c0;
+  int p2 = a.c0 * b.c2 + a.c1 * b.c1 + a.c2 * b.c0;
+  int p3 = a.c1 * b.c2 + a.c2 * b.c1;
+  int p4 = a.c2 * b.c2;
+  return Gf27{(p0 + 2 * p3) % 3, (p1 + p3 + 2 * p4) % 3, (p2 + p4) % 3};
+}
+
+// Quadratic character by Euler's criterion: e^((27-1)/2) is 1 on squares, -1 otherwise.
+__host__ __device__ constexpr int gf_character(int e) {
+  if (e == 0) return 0;
+  Gf27 base = gf_from_index(e);
+  Gf27 acc = Gf27{1, 0, 0};
+  for (int i = 0; i < 13; ++i) acc = gf_prod(acc, base);
+  return gf_to_index(acc) == 1 ? 1 : -1;
+}
+
+// H28[r][c]: first row all +1, first column +1 then -1, core I + chi(r - c).
+__host__ __device__ constexpr int paley28_entry(int r, int c) {
+  if (r == 0) return 1;
+  if (c == 0) return -1;
+  if (r == c) return 1;
+  return gf_character(gf_to_index(gf_diff(gf_from_index(r - 1), gf_from_index(c - 1))));
+}
+
+struct Paley28Table {
+  float v[28][28];
+};
+
+constexpr Paley28Table make_paley28_table() {
+  Paley28Table t{};
+  for (int r = 0; r < 28; ++r)
+    for (int c = 0; c < 28; ++c) t.v[r][c] = float(paley28_entry(r, c));
+  return t;
+}
+
+__constant__ Paley28Table c_paley28 = make_paley28_table();
+
+// ---------------------------------------------------------------------------
+// Small device helpers
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Step size of Eq. 1's symmetric form with a clip ratio: clip * max / 7.
+__device__ __forceinline__ float step_from_absmax(float amax, float clip) {
+  return amax == 0.0f ? 1.0f : __fdiv_rn(__fmul_rn(clip, amax), 7.0f);
+}
+
+__device__ __forceinline__ void unpack8_f16(const uint4& raw, float* f) {
+  const __half2* h = reinterpret_cast<const __half2*>(&raw);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float2 t = __half22float2(h[i]);
+    f[2 * i] = t.x;
+    f[2 * i + 1] = t.y;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Generic kernel: one CTA per row.
+// ---------------------------------------------------------------------------
+constexpr int kGenericThreads = 256;
+
+template <bool kQuant>
+__global__ void __launch_bounds__(kGenericThreads)
+rotate_generic_kernel(const __half* __restrict__ X, int64_t ldx, int K, int base, int n, int logn,
+                      const float* __restrict__ pre, float inv_sqrt_k, float clip,
+                      uint8_t* __restrict__ q_out, float* __restrict__ step_out,
+                      float* __restrict__ y_out) {
+  extern __shared__ __align__(16) float row[];
+  __shared__ float red[kGenericThreads / 32];
+  const int tid = threadIdx.x;
+  const int64_t m = blockIdx.x;
+  const __half* x = X + m * ldx;
+
+  for (int c = tid; c < K / 8; c += kGenericThreads) {
+    uint4 raw = *reinterpret_cast<const uint4*>(x + c * 8);
+    float f[8];
+    unpack8_f16(raw, f);
+    if (pre != nullptr) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) f[i] *= pre[c * 8 + i];
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) row[c * 8 + i] = f[i];
+  }
+  __syncthreads();
+
+  // Walsh butterflies on the low `logn` index bits, up to three bits per pass.
+  for (int s = 0; s < logn; s += 3) {
+    const int nb = min(3, logn - s);
+    const int cnt = 1 << nb;
+    const int groups = K >> nb;
+    for (int v = tid; v < groups; v += kGenericThreads) {
+      const int lo = v & ((1 << s) - 1);
+      const int hi = v >> s;
+      const int idx0 = lo | (hi << (s + nb));
+      float e[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) e[i] = (i < cnt) ? row[idx0 + (i << s)] : 0.0f;
+#pragma unroll
+      for (int h = 1; h < 8; h <<= 1) {
+        if (h < cnt) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            if ((i & h) == 0) {
+              float a = e[i], b = e[i + h];
+              e[i] = a + b;
+              e[i + h] = a - b;
+            }
+          }
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        if (i < cnt) row[idx0 + (i << s)] = e[i];
+    }
+    __syncthreads();
+  }
+
+  // Order-28 factor on the slow index a of j = a * n + b:  y[a'] = sum_a x[a] H28[a][a'].
+  if (base == 28) {
+    for (int b = tid; b < n; b += kGenericThreads) {
+      float xin[28], yv[28];
+#pragma unroll
+      for (int a = 0; a < 28; ++a) xin[a] = row[a * n + b];
+#pragma unroll
+      for (int c = 0; c < 28; ++c) {
+        float acc = 0.0f;
+#pragma unroll
+        for (int a = 0; a < 28; ++a) acc = fmaf(xin[a], c_paley28.v[a][c], acc);
+        yv[c] = acc;
+      }
+#pragma unroll
+      for (int c = 0; c < 28; ++c) row[c * n + b] = yv[c];
+    }
+    __syncthreads();
+  }
+
+  if (!kQuant) {
+    float* y = y_out + m * int64_t(K);
+    for (int j = tid; j < K; j += kGenericThreads) y[j] = row[j] * inv_sqrt_k;
+    return;
+  }
+
+  float amax = 0.0f;
+  for (int j = tid; j < K; j += kGenericThreads) {
+    float v = row[j] * inv_sqrt_k;
+    row[j] = v;
+    amax = fmaxf(amax, fabsf(v));
+  }
+  amax = warp_max(amax);
+  if ((tid & 31) == 0) red[tid >> 5] = amax;
+  __syncthreads();
+  amax = red[0];
+#pragma unroll
+  for (int w = 1; w < kGenericThreads / 32; ++w) amax = fmaxf(amax, red[w]);
+  const float step = step_from_absmax(amax, clip);
+  if (tid == 0) step_out[m] = step;
+
+  uint32_t* q = reinterpret_cast<uint32_t*>(q_out + m * int64_t(K / 2));
+  for (int c = tid; c < K / 8; c += kGenericThreads) {
+    uint32_t word = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      float t = rintf(__fdiv_rn(row[c * 8 + i], step));
+      t = fminf(fmaxf(t, -8.0f), 7.0f);
+      word |= (uint32_t(int(t)) & 0xFu) << (4 * i);
+    }
+    q[c] = word;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// K = 4096.  A CTA holds kRowsPerCta rows, 64 threads (two warps) per row.
+//
+// Index bits of a row position j (12 bits):  i = j[0:3), t = j[3:9), g = j[9:12).
+//   phase 1  thread t loads the eight 16-byte chunks (g, t): values (g, i);
+//            butterflies on the bits of i and g (6 stages, in registers).
+//   transpose through shared memory: [t][g*8+i], row pitch 68 floats.
+//   phase 2  thread (g, i) holds the 64 values over t; butterflies on the six
+//            bits of t.  1/sqrt(4096) = 2^-6 is folded into `pre` (exact).
+//   absmax over the row, step size, rounding by the 1.5 * 2^23 trick, then the
+//   codes travel between the lanes of a row group so that each lane ends up
+//   with whole 32-bit words of packed output.
+// ---------------------------------------------------------------------------
+constexpr int kW4096Rows = 4;
+constexpr int kW4096Pitch = 68;  // floats per t-row in shared memory (64 + 4 pad)
+
+__device__ __forceinline__ void group_barrier(int group) {
+  asm volatile("bar.sync %0, 64;" ::"r"(group + 1) : "memory");
+}
+
+template <int N>
+__device__ __forceinline__ void butterflies_inplace(float* v) {
+#pragma unroll
+  for (int h = 1; h < N; h <<= 1) {
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+      if ((i & h) == 0) {
+        float a = v[i], b = v[i + h];
+        v[i] = a + b;
+        v[i + h] = a - b;
+      }
+    }
+  }
+}
+
+template <bool kQuant, bool kHasPre>
+__global__ void __launch_bounds__(kW4096Rows * 64)
+walsh4096_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
+                 const float* __restrict__ pre, float clip,
+                 uint8_t* __restrict__ q_out, float* __restrict__ step_out,
+                 float* __restrict__ y_out) {
+  extern __shared__ __align__(16) float smem[];
+  __shared__ float red[kW4096Rows][2];
+  const int group = threadIdx.x >> 6;
+  const int t = threadIdx.x & 63;
+  const int lane = threadIdx.x & 31;
+  const int64_t m = int64_t(blockIdx.x) * kW4096Rows + group;
+  if (m >= M) return;  // whole row group leaves together; only group barriers are used
+  float* tile = smem + group * (64 * kW4096Pitch);
+
+  float v[64];
+  {
+    const __half* x = X + m * ldx;
+    uint4 raw[8];
+#pragma unroll
+    for (int g = 0; g < 8; ++g) raw[g] = __ldg(reinterpret_cast<const uint4*>(x + g * 512 + t * 8));
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+      unpack8_f16(raw[g], &v[g * 8]);
+      if (kHasPre) {
+        const float4 p0 = __ldg(reinterpret_cast<const float4*>(pre + g * 512 + t * 8));
+        const float4 p1 = __ldg(reinterpret_cast<const float4*>(pre + g * 512 + t * 8 + 4));
+        v[g * 8 + 0] *= p0.x * 0.015625f; v[g * 8 + 1] *= p0.y * 0.015625f;
+        v[g * 8 + 2] *= p0.z * 0.015625f; v[g * 8 + 3] *= p0.w * 0.015625f;
+        v[g * 8 + 4] *= p1.x * 0.015625f; v[g * 8 + 5] *= p1.y * 0.015625f;
+        v[g * 8 + 6] *= p1.z * 0.015625f; v[g * 8 + 7] *= p1.w * 0.015625f;
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[g * 8 + i] *= 0.015625f;
+      }
+    }
+  }
+  butterflies_inplace<64>(v);  // v index = g * 8 + i: bits of i, then bits of g
+
+  // transpose: thread t writes its 64 values as one padded row
+  {
+    float4* dst = reinterpret_cast<float4*>(tile + t * kW4096Pitch);
+#pragma unroll
+    for (int c = 0; c < 16; ++c) dst[c] = make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+  }
+  group_barrier(group);
+  // thread gi = t now owns position (g, i) = (t >> 3, t & 7) for all 64 values of the t-bits
+#pragma unroll
+  for (int u = 0; u < 64; ++u) v[u] = tile[u * kW4096Pitch + t];
+  butterflies_inplace<64>(v);
+
+  const int gi_g = t >> 3, gi_i = t & 7;
+  if (!kQuant) {
+    float* y = y_out + m * 4096;
+#pragma unroll
+    for (int u = 0; u < 64; ++u) y[gi_g * 512 + u * 8 + gi_i] = v[u];
+    return;
+  }
+
+  float amax = 0.0f;
+#pragma unroll
+  for (int u = 0; u < 64; ++u) amax = fmaxf(amax, fabsf(v[u]));
+  amax = warp_max(amax);
+  if (lane == 0) red[group][t >> 5] = amax;
+  group_barrier(group);
+  amax = fmaxf(red[group][0], red[group][1]);
+  const float step = step_from_absmax(amax, clip);
+  if (t == 0) step_out[m] = step;
+  const float inv = __frcp_rn(step);
+
+  // Round to nearest even and bias by 8: the low byte of the float's bit
+  // pattern is code + 8 in [0, 15].
+  const float kMagic = 12582912.0f + 8.0f;  // 1.5 * 2^23 + 8
+  uint32_t spread[16];                      // four codes per word, one per byte
+#pragma unroll
+  for (int c = 0; c < 16; ++c) {
+    uint32_t r[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      float q = fmaf(v[4 * c + k], inv, kMagic);
+      q = fminf(fmaxf(q, 12582912.0f), 12582912.0f + 15.0f);
+      r[k] = __float_as_uint(q);
+    }
+    const uint32_t lo = __byte_perm(r[0], r[1], 0x0040);  // bytes: r0.b0, r1.b0
+    const uint32_t hi = __byte_perm(r[2], r[3], 0x0040);
+    spread[c] = __byte_perm(lo, hi, 0x5410);
+  }
+  // Lanes 2p and 2p+1 hold the even and odd position of each byte.  The even
+  // lane finishes the words with even c, the odd lane those with odd c.
+  const bool odd = (gi_i & 1) != 0;
+  uint32_t word[8];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    const uint32_t give = odd ? spread[2 * c] : spread[2 * c + 1];
+    const uint32_t keep = odd ? spread[2 * c + 1] : spread[2 * c];
+    const uint32_t got = __shfl_xor_sync(0xffffffffu, give, 1);
+    const uint32_t lo_n = odd ? got : keep;   // even position -> low nibble
+    const uint32_t hi_n = odd ? keep : got;
+    word[c] = (lo_n | (hi_n << 4)) ^ 0x88888888u;  // offset binary -> two's complement
+  }
+  // word[c] of lane (g, i) holds, for u = 4 * (2c + odd) + k (k = byte), the
+  // output byte at  g * 256 + u * 4 + (i >> 1).  A 4 x 4 byte transpose among
+  // the lanes i>>1 = 0..3 turns these into aligned 32-bit words.
+  const int r = gi_i >> 1;
+  const uint32_t sel1 = (r & 1) ? 0x3715u : 0x6240u;  // step 1 selector (own = a, partner = b)
+  const uint32_t sel2 = (r & 2) ? 0x3276u : 0x5410u;  // step 2 selector
+  uint32_t* q = reinterpret_cast<uint32_t*>(q_out + m * 2048);
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    uint32_t w = word[c];
+    uint32_t p = __shfl_xor_sync(0xffffffffu, w, 2);
+    // r even: [own.k0, p.k0, own.k2, p.k2];  r odd: [p.k1, own.k1, p.k3, own.k3]
+    w = __byte_perm(w, p, sel1);
+    p = __shfl_xor_sync(0xffffffffu, w, 4);
+    // r < 2: [own.b0, own.b1, p.b0, p.b1];  r >= 2: [p.b2, p.b3, own.b2, own.b3]
+    w = __byte_perm(w, p, sel2);
+    const int u = 4 * (2 * c + (odd ? 1 : 0)) + r;
+    q[gi_g * 64 + u] = w;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------
+static int check_rows(const void* X, int64_t rows, int64_t K, int64_t ld, int* base, int* n, int* logn) {
+  if (rows < 0 || K <= 0) return SMOOTHROT_INVALID_ARG;
+  if (!split_order(K, base, n, logn)) return SMOOTHROT_UNSUPPORTED_K;
+  if (rows == 0) return SMOOTHROT_OK;
+  if (X == nullptr || ld < K) return SMOOTHROT_INVALID_ARG;
+  if (!aligned16(X) || (ld % 8) != 0) return SMOOTHROT_BAD_ALIGNMENT;
+  if (rows > 0x7fffffffLL) return SMOOTHROT_INVALID_ARG;
+  return SMOOTHROT_OK;
+}
+
+template <bool kQuant>
+static int launch_rotate(const void* X, int64_t rows, int64_t K, int64_t ld, const float* pre, float clip,
+                         uint8_t* q_out, float* step_out, float* y_out, cudaStream_t stream) {
+  int base = 0, n = 0, logn = 0;
+  int rc = check_rows(X, rows, K, ld, &base, &n, &logn);
+  if (rc != SMOOTHROT_OK || rows == 0) return rc;
+  const __half* x = static_cast<const __half*>(X);
+  if (K == 4096) {
+    const size_t smem = size_t(kW4096Rows) * 64 * kW4096Pitch * sizeof(float);
+    auto kern = pre ? walsh4096_kernel<kQuant, true> : walsh4096_kernel<kQuant, false>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
+      return SMOOTHROT_CUDA_ERROR;
+    const unsigned grid = unsigned((rows + kW4096Rows - 1) / kW4096Rows);
+    kern<<<grid, kW4096Rows * 64, smem, stream>>>(x, ld, rows, pre, clip, q_out, step_out, y_out);
+    count_launch();
+    return launch_status();
+  }
+  const size_t smem = size_t(K) * sizeof(float);
+  auto kern = rotate_generic_kernel<kQuant>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
+    return SMOOTHROT_CUDA_ERROR;
+  const float inv_sqrt_k = float(1.0 / sqrt(double(K)));
+  kern<<<unsigned(rows), kGenericThreads, smem, stream>>>(x, ld, int(K), base, n, logn, pre, inv_sqrt_k, clip,
+                                                           q_out, step_out, y_out);
+  count_launch();
+  return launch_status();
+}
+
+static int quantize_entry(const void* X, int64_t rows, int64_t K, int64_t ld, const float* pre, float clip,
+                          uint8_t* q_out, float* step_out, void* stream) {
+  if (!(clip > 0.0f) || clip > 1.0f) return SMOOTHROT_INVALID_ARG;
+  if (rows > 0 && (q_out == nullptr || step_out == nullptr)) return SMOOTHROT_INVALID_ARG;
+  if (rows > 0 && (!aligned16(q_out) || (pre != nullptr && !aligned16(pre)))) return SMOOTHROT_BAD_ALIGNMENT;
+  return launch_rotate<true>(X, rows, K, ld, pre, clip, q_out, step_out, nullptr,
+                             static_cast<cudaStream_t>(stream));
+}
+
+}  // namespace smoothrot
+
+extern "C" {
+
+int smoothrot_fuse_weights(const void* W_f16, int64_t N, int64_t K, int64_t ldw, const float* pre,
+                           float clip_w, uint8_t* Wq_out, float* dw_out, void* stream) {
+  return smoothrot::quantize_entry(W_f16, N, K, ldw, pre, clip_w, Wq_out, dw_out, stream);
+}
+
+int smoothrot_quant_act(const void* X_f16, int64_t M, int64_t K, int64_t ldx, const float* pre,
+                        float clip_a, uint8_t* Xq_out, float* dx_out, void* stream) {
+  return smoothrot::quantize_entry(X_f16, M, K, ldx, pre, clip_a, Xq_out, dx_out, stream);
+}
+
+int smoothrot_debug_hadamard(const void* X_f16, int64_t M, int64_t K, int64_t ldx, const float* pre,
+                             float* Y_f32, void* stream) {
+  if (M > 0 && Y_f32 == nullptr) return SMOOTHROT_INVALID_ARG;
+  if (M > 0 && pre != nullptr && !smoothrot::aligned16(pre)) return SMOOTHROT_BAD_ALIGNMENT;
+  return smoothrot::launch_rotate<false>(X_f16, M, K, ldx, pre, 1.0f, nullptr, nullptr, Y_f32,
+                                         static_cast<cudaStream_t>(stream));
+}
+
+int smoothrot_paley28(int8_t* out_host) {
+  if (out_host == nullptr) return SMOOTHROT_INVALID_ARG;
+  for (int r = 0; r < 28; ++r)
+    for (int c = 0; c < 28; ++c) out_host[r * 28 + c] = int8_t(smoothrot::paley28_entry(r, c));
+  return SMOOTHROT_OK;
+}
+
+}  // extern "C"

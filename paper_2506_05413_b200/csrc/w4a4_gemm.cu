@@ -1,0 +1,669 @@
+// W4A4 GEMM of libsmoothrot:  acc[m][n] = sum_k Xq[m][k] Wq[n][k]  on packed
+// 4-bit codes, with the dequantization  Y = fp16(acc * dx[m] * dw[n])  fused
+// into the epilogue (Eq. 2's product on Eq. 1's integer codes, then Eq. 1's
+// dequantizer on both factors).
+//
+// sm_100a has no 4-bit integer MMA, so the codes are widened to int8 on the
+// way to the tensor core:
+//
+//   TMA (cp.async.bulk.tensor, 64-byte swizzle) brings 64 packed bytes per
+//   row and k-block into shared memory;
+//   "widen" warps read 16 packed bytes and write two 16-byte int8 vectors
+//   (w & 0xF0F0F0F0 and (w << 4) & 0xF0F0F0F0: each byte lane is 16 * code in
+//   two's complement, no sign extension needed) into the 128-byte-swizzled
+//   K-major layout tcgen05.mma reads.  Both operands get the same permutation
+//   of k inside a k-block, which a dot product does not see;
+//   one thread issues tcgen05.mma.kind::i8 (128 x BN x 32) with the int32
+//   accumulator in tensor memory; accumulators are 256 * acc, exact, and
+//   |256 * acc| <= K * 128 * 128 < 2^31 for K <= 65536;
+//   four epilogue warps read the accumulator with tcgen05.ld, shift by 8,
+//   scale and store, while the next tile's main loop runs on the other half
+//   of tensor memory.
+//
+// The kernel is persistent (one CTA per SM, tiles handed out round-robin).
+// For M < 128 tokens the roles of the operands are swapped (output channels on
+// the 128-row MMA axis, tokens on the N axis) and K is split across CTAs;
+// the int32 partial sums go to the caller's workspace and a second kernel
+// adds them and dequantizes.
+//
+// Every wait on an mbarrier is bounded in wall time; a wait that runs out
+// sets a device status word, raises a CTA-wide abort flag and the kernel
+// winds down normally.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace smoothrot {
+namespace gemm {
+
+constexpr int kBM = 128;            // MMA M: rows of the A side per tile
+constexpr int kPackedRow = 64;      // packed bytes per row and k-block
+constexpr int kWideRow = 128;       // int8 bytes per row and k-block (= codes per k-block)
+constexpr int kWidenWarps = 8;
+constexpr int kEpiWarps = 4;
+constexpr int kThreads = 32 * (2 + kWidenWarps + kEpiWarps);
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
+
+__device__ int g_device_status = 0;
+
+enum TimeoutSite { kSiteProducer = 1, kSiteWidenFull = 2, kSiteWidenEmpty = 3, kSiteMmaAcc = 4,
+                   kSiteMmaWide = 5, kSiteEpilogue = 6 };
+
+template <int BN>
+struct Tile {
+  static constexpr int kWideStages = BN >= 256 ? 2 : (BN >= 128 ? 3 : 4);
+  static constexpr int kPackedStages = BN >= 256 ? 4 : (BN >= 128 ? 4 : 6);
+  static constexpr int kWideA = kBM * kWideRow, kWideB = BN * kWideRow;
+  static constexpr int kPackedA = kBM * kPackedRow, kPackedB = BN * kPackedRow;
+  // kPackedB may be below 1024 bytes (BN = 16): round stage parts up to 1024 so
+  // that every tile base keeps the alignment the swizzle patterns assume.
+  static constexpr int kPackedBPad = (kPackedB + 1023) / 1024 * 1024;
+  static constexpr int kWideBPad = (kWideB + 1023) / 1024 * 1024;
+  static constexpr int kWideStageBytes = kWideA + kWideBPad;
+  static constexpr int kPackedStageBytes = kPackedA + kPackedBPad;
+  static constexpr int kNumBarriers = 2 * kWideStages + 2 * kPackedStages + 4;
+  static constexpr int kSmemBytes = 1024 /*alignment slack*/ + kWideStages * kWideStageBytes +
+                                    kPackedStages * kPackedStageBytes + kNumBarriers * 8 + 16;
+  static constexpr int kTmemCols = (2 * BN) < 32 ? 32 : 2 * BN;  // two accumulators, power of two
+};
+
+// ---------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return uint32_t(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Waits for the barrier phase with the given parity, at most kWaitLimitNs.
+// Returns false if the wait ran out or another role of this CTA gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int site) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (uint32_t spin = 1;; ++spin) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((spin & 63u) == 0u) {
+      if (*abort_flag != 0) return false;
+      if (global_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        atomicCAS(&g_device_status, 0, site);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+
+__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tcgen05_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void mma_i8(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                       uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+__device__ __forceinline__ void tmem_load32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_load16(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of
+// 128 bytes, groups of 8 rows 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_desc_sw128(uint32_t smem_addr) {
+  const uint32_t lo = ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16);
+  const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+  return (uint64_t(hi) << 32) | lo;
+}
+
+// Instruction descriptor: int8 x int8 -> int32, both operands K-major, M = 128.
+__host__ __device__ constexpr uint32_t make_idesc_i8(int n) {
+  return (2u << 4) | (1u << 7) | (1u << 10) | (uint32_t(n >> 3) << 17) | (uint32_t(kBM >> 4) << 24);
+}
+
+// ---------------------------------------------------------------------------
+// Kernel parameters
+// ---------------------------------------------------------------------------
+struct Params {
+  int rows_a, rows_b;     // valid rows of the A-side and B-side matrices
+  int tiles_a, tiles_b;   // tile counts
+  int kblocks;            // K / 128
+  int splits;             // k-splits (1 = none)
+  int swapped;            // 0: A side = tokens (Xq), B side = channels (Wq); 1: the reverse
+  int M, N;               // logical output shape
+  const float* dx;        // [M]
+  const float* dw;        // [N]
+  __half* Y;              // [M x ldy] (direct dequantized output) or nullptr
+  int64_t ldy;
+  int32_t* acc_out;       // [splits][M][N] int32 (debug export or split-K partials) or nullptr
+};
+
+// Writes 32 consecutive accumulator columns [c0, c0 + 32) of A-side row `a`.
+template <int NCOLS>
+__device__ __forceinline__ void store_columns(const Params& p, int a, int b0, int split, const uint32_t* r) {
+  if (a >= p.rows_a) return;
+  if (!p.swapped) {
+    const int m = a;
+    if (p.Y != nullptr) {
+      const float sx = __ldg(p.dx + m);
+      __half* y = p.Y + int64_t(m) * p.ldy + b0;
+#pragma unroll
+      for (int j = 0; j < NCOLS; j += 8) {
+        if (b0 + j + 8 <= p.rows_b) {
+          const float4 w0 = __ldg(reinterpret_cast<const float4*>(p.dw + b0 + j));
+          const float4 w1 = __ldg(reinterpret_cast<const float4*>(p.dw + b0 + j + 4));
+          const float ws[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+          uint4 out;
+          __half2* h = reinterpret_cast<__half2*>(&out);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const float v0 = float(int32_t(r[j + 2 * q]) >> 8) * (sx * ws[2 * q]);
+            const float v1 = float(int32_t(r[j + 2 * q + 1]) >> 8) * (sx * ws[2 * q + 1]);
+            h[q] = __floats2half2_rn(v0, v1);
+          }
+          *reinterpret_cast<uint4*>(y + j) = out;
+        }
+      }
+    } else {
+      int32_t* o = p.acc_out + (int64_t(split) * p.M + m) * p.N + b0;
+#pragma unroll
+      for (int j = 0; j < NCOLS; j += 4) {
+        if (b0 + j + 4 <= p.rows_b) {
+          int4 v = make_int4(int32_t(r[j]) >> 8, int32_t(r[j + 1]) >> 8, int32_t(r[j + 2]) >> 8,
+                             int32_t(r[j + 3]) >> 8);
+          *reinterpret_cast<int4*>(o + j) = v;
+        }
+      }
+    }
+  } else {
+    const int n = a;  // output channel; columns are tokens
+    if (p.Y != nullptr) {
+      const float sw = __ldg(p.dw + n);
+#pragma unroll
+      for (int j = 0; j < NCOLS; ++j) {
+        const int m = b0 + j;
+        if (m < p.rows_b) {
+          const float v = float(int32_t(r[j]) >> 8) * (__ldg(p.dx + m) * sw);
+          p.Y[int64_t(m) * p.ldy + n] = __float2half_rn(v);
+        }
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < NCOLS; ++j) {
+        const int m = b0 + j;
+        if (m < p.rows_b) p.acc_out[(int64_t(split) * p.M + m) * p.N + n] = int32_t(r[j]) >> 8;
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// The kernel
+// ---------------------------------------------------------------------------
+template <int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+w4a4_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                 const Params p) {
+  using T = Tile<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t base = (raw_addr + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - raw_addr);
+
+  const uint32_t wide_base = base;
+  const uint32_t packed_base = wide_base + T::kWideStages * T::kWideStageBytes;
+  const uint32_t bar_base = packed_base + T::kPackedStages * T::kPackedStageBytes;
+  // barrier order: wide_full[WS], wide_empty[WS], pk_full[PS], pk_empty[PS], acc_full[2], acc_empty[2]
+  auto wide_full = [&](int s) { return bar_base + 8u * s; };
+  auto wide_empty = [&](int s) { return bar_base + 8u * (T::kWideStages + s); };
+  auto pk_full = [&](int s) { return bar_base + 8u * (2 * T::kWideStages + s); };
+  auto pk_empty = [&](int s) { return bar_base + 8u * (2 * T::kWideStages + T::kPackedStages + s); };
+  auto acc_full = [&](int s) { return bar_base + 8u * (2 * T::kWideStages + 2 * T::kPackedStages + s); };
+  auto acc_empty = [&](int s) { return bar_base + 8u * (2 * T::kWideStages + 2 * T::kPackedStages + 2 + s); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + (bar_base - base) + 8 * T::kNumBarriers);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < T::kWideStages; ++s) {
+      mbar_init(wide_full(s), kWidenWarps);
+      mbar_init(wide_empty(s), 1);
+    }
+    for (int s = 0; s < T::kPackedStages; ++s) {
+      mbar_init(pk_full(s), 1);
+      mbar_init(pk_empty(s), kWidenWarps);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(acc_full(s), 1);
+      mbar_init(acc_empty(s), kEpiWarps);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async();
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(tmem_slot)), "r"(uint32_t(T::kTmemCols)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int total_tiles = p.tiles_a * p.tiles_b * p.splits;
+  const int kb_per_split = p.kblocks / p.splits;  // host guarantees divisibility
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int ta = tile % p.tiles_a;
+        const int rest = tile / p.tiles_a;
+        const int tb = rest % p.tiles_b;
+        const int split = rest / p.tiles_b;
+        const int kb0 = split * kb_per_split;
+        for (int kb = kb0; kb < kb0 + kb_per_split; ++kb, ++it) {
+          const int s = it % T::kPackedStages;
+          const uint32_t ph = (it / T::kPackedStages) & 1u;
+          if (!mbar_wait(pk_empty(s), ph ^ 1u, abort_flag, kSiteProducer)) { ok = false; break; }
+          mbar_expect_tx(pk_full(s), uint32_t(T::kPackedA + T::kPackedB));
+          const uint32_t dst = packed_base + s * T::kPackedStageBytes;
+          tma_load_2d(dst, &map_a, pk_full(s), kb * kPackedRow, ta * kBM);
+          tma_load_2d(dst + T::kPackedA, &map_b, pk_full(s), kb * kPackedRow, tb * BN);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_i8(BN);
+      uint32_t it = 0, local_tile = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local_tile) {
+        const int ab = local_tile & 1;
+        const uint32_t aph = (local_tile >> 1) & 1u;
+        if (!mbar_wait(acc_empty(ab), aph ^ 1u, abort_flag, kSiteMmaAcc)) break;
+        tcgen05_fence_after();
+        const uint32_t tmem_d = tmem_base + uint32_t(ab * BN);
+        for (int kb = 0; kb < kb_per_split; ++kb, ++it) {
+          const int s = it % T::kWideStages;
+          const uint32_t ph = (it / T::kWideStages) & 1u;
+          if (!mbar_wait(wide_full(s), ph, abort_flag, kSiteMmaWide)) { ok = false; break; }
+          tcgen05_fence_after();
+          const uint32_t a_addr = wide_base + s * T::kWideStageBytes;
+          const uint64_t da = make_desc_sw128(a_addr);
+          const uint64_t db = make_desc_sw128(a_addr + T::kWideA);
+#pragma unroll
+          for (int k4 = 0; k4 < 4; ++k4) {
+            // 32 int8 = 32 bytes further along K inside the swizzle atom: +2 in 16-byte units
+            mma_i8(tmem_d, da + uint64_t(2 * k4), db + uint64_t(2 * k4), idesc, (kb > 0 || k4 > 0) ? 1u : 0u);
+          }
+          tcgen05_commit(wide_empty(s));
+        }
+        if (ok) tcgen05_commit(acc_full(ab));
+      }
+    }
+  } else if (warp < 2 + kWidenWarps) {
+    // ------------------------------------------------------------ widen warps
+    const int w = warp - 2;
+    const int r = lane & 7;    // row inside an 8-row group
+    const int c = lane >> 3;   // 16-byte chunk of the packed row (0..3)
+    constexpr int kGroupsA = kBM / 8;
+    constexpr int kGroups = (kBM + BN) / 8;
+    uint32_t it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      for (int kb = 0; kb < kb_per_split; ++kb, ++it) {
+        const int ps = it % T::kPackedStages;
+        const uint32_t pph = (it / T::kPackedStages) & 1u;
+        const int ws = it % T::kWideStages;
+        const uint32_t wph = (it / T::kWideStages) & 1u;
+        if (!mbar_wait(pk_full(ps), pph, abort_flag, kSiteWidenFull)) { ok = false; break; }
+        if (!mbar_wait(wide_empty(ws), wph ^ 1u, abort_flag, kSiteWidenEmpty)) { ok = false; break; }
+        const uint32_t pk = packed_base + ps * T::kPackedStageBytes;
+        const uint32_t wd = wide_base + ws * T::kWideStageBytes;
+#pragma unroll 2
+        for (int g = w; g < kGroups; g += kWidenWarps) {
+          // operand-local row and the two tile bases
+          const bool is_b = g >= kGroupsA;
+          const int row = (is_b ? g - kGroupsA : g) * 8 + r;
+          const uint32_t src = (is_b ? pk + T::kPackedA : pk) + row * kPackedRow + ((c ^ ((row >> 1) & 3)) << 4);
+          const uint32_t dst_row = (is_b ? wd + T::kWideA : wd) + row * kWideRow;
+          uint32_t x0, x1, x2, x3;
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                       : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3) : "r"(src) : "memory");
+          const uint32_t lo_dst = dst_row + (((2 * c) ^ (row & 7)) << 4);
+          const uint32_t hi_dst = dst_row + (((2 * c + 1) ^ (row & 7)) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                       ::"r"(lo_dst), "r"((x0 << 4) & 0xF0F0F0F0u), "r"((x1 << 4) & 0xF0F0F0F0u),
+                         "r"((x2 << 4) & 0xF0F0F0F0u), "r"((x3 << 4) & 0xF0F0F0F0u) : "memory");
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                       ::"r"(hi_dst), "r"(x0 & 0xF0F0F0F0u), "r"(x1 & 0xF0F0F0F0u),
+                         "r"(x2 & 0xF0F0F0F0u), "r"(x3 & 0xF0F0F0F0u) : "memory");
+        }
+        fence_proxy_async();   // make the generic-proxy stores visible to the tensor core
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(wide_full(ws));
+          mbar_arrive(pk_empty(ps));
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue warps
+    const int e = warp & 3;  // tensor-memory lane quadrant this warp may read
+    uint32_t local_tile = 0;
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++local_tile) {
+      const int ta = tile % p.tiles_a;
+      const int rest = tile / p.tiles_a;
+      const int tb = rest % p.tiles_b;
+      const int split = rest / p.tiles_b;
+      const int ab = local_tile & 1;
+      const uint32_t aph = (local_tile >> 1) & 1u;
+      if (!mbar_wait(acc_full(ab), aph, abort_flag, kSiteEpilogue)) break;
+      tcgen05_fence_after();
+      const int a = ta * kBM + e * 32 + lane;
+      const uint32_t taddr = tmem_base + (uint32_t(e * 32) << 16) + uint32_t(ab * BN);
+      if constexpr (BN >= 32) {
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          uint32_t regs[32];
+          tmem_load32(taddr + c0, regs);
+          tmem_wait_ld();
+          store_columns<32>(p, a, tb * BN + c0, split, regs);
+          __syncwarp();
+        }
+      } else {
+        uint32_t regs[16];
+        tmem_load16(taddr, regs);
+        tmem_wait_ld();
+        store_columns<16>(p, a, tb * BN, split, regs);
+        __syncwarp();
+      }
+      tcgen05_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty(ab));
+    }
+  }
+
+  tcgen05_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tcgen05_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
+                 ::"r"(tmem_base), "r"(uint32_t(T::kTmemCols)) : "memory");
+  }
+}
+
+// Sums the split-K partials and applies the dequantization (or writes the int32 sum).
+__global__ void splitk_reduce_kernel(const int32_t* __restrict__ part, int splits, int M, int N,
+                                     const float* __restrict__ dx, const float* __restrict__ dw,
+                                     __half* __restrict__ Y, int64_t ldy, int32_t* __restrict__ acc_out) {
+  const int64_t idx = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+  const int64_t total = int64_t(M) * N;
+  if (idx >= total) return;
+  int32_t sum = 0;
+  for (int s = 0; s < splits; ++s) sum += part[int64_t(s) * total + idx];
+  const int m = int(idx / N), n = int(idx % N);
+  if (Y != nullptr) {
+    Y[int64_t(m) * ldy + n] = __float2half_rn(float(sum) * (dx[m] * dw[n]));
+  } else {
+    acc_out[idx] = sum;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------
+struct Plan {
+  bool swapped;
+  int bn;
+  int splits;
+};
+
+static int sm_count() {
+  static int cached = 0;
+  if (cached == 0) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+      cached = n;
+    else
+      return 148;
+  }
+  return cached;
+}
+
+static Plan make_plan(int64_t M, int64_t N, int64_t K) {
+  Plan pl{};
+  const int kblocks = int(K / kWideRow);
+  if (M >= 128) {
+    pl.swapped = false;
+    pl.bn = (N >= 256) ? 256 : (N > 64 ? 128 : 64);
+    pl.splits = 1;
+    return pl;
+  }
+  pl.swapped = true;
+  pl.bn = M <= 16 ? 16 : (M <= 32 ? 32 : (M <= 64 ? 64 : 128));
+  const int tiles = int((N + kBM - 1) / kBM);
+  int want = (sm_count() + tiles - 1) / tiles;
+  if (want < 1) want = 1;
+  int splits = 1;
+  // largest divisor of kblocks that does not exceed `want` and leaves >= 4 k-blocks per split
+  for (int s = 1; s <= kblocks && s <= want; ++s)
+    if (kblocks % s == 0 && kblocks / s >= 4) splits = s;
+  pl.splits = splits;
+  return pl;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// 2-D map over a packed matrix [rows x K/2] bytes, box = 64 bytes x box_rows, 64-byte swizzle.
+static bool make_map(CUtensorMap* map, const uint8_t* ptr, int64_t rows, int64_t K, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  const cuuint64_t dims[2] = {cuuint64_t(K / 2), cuuint64_t(rows)};
+  const cuuint64_t strides[1] = {cuuint64_t(K / 2)};
+  const cuuint32_t box[2] = {cuuint32_t(kPackedRow), cuuint32_t(box_rows)};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN>
+static int launch_tile(const CUtensorMap& ma, const CUtensorMap& mb, const Params& p, cudaStream_t st) {
+  auto kern = w4a4_gemm_kernel<BN>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Tile<BN>::kSmemBytes) != cudaSuccess)
+    return SMOOTHROT_CUDA_ERROR;
+  const int total = p.tiles_a * p.tiles_b * p.splits;
+  const int grid = total < sm_count() ? total : sm_count();
+  kern<<<grid, kThreads, Tile<BN>::kSmemBytes, st>>>(ma, mb, p);
+  count_launch();
+  return launch_status();
+}
+
+static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq, const float* dw, int64_t N,
+               int64_t K, __half* Y, int64_t ldy, int32_t* acc_out, void* workspace, size_t workspace_bytes,
+               cudaStream_t st) {
+  if (M < 0 || N < 0 || K <= 0) return SMOOTHROT_INVALID_ARG;
+  if (K % kWideRow != 0 || K > 65536) return SMOOTHROT_UNSUPPORTED_K;
+  if (N % 8 != 0) return SMOOTHROT_INVALID_ARG;
+  if (M == 0 || N == 0) return SMOOTHROT_OK;
+  if (M > 0x7fffffffLL / 2 || N > 0x7fffffffLL / 2) return SMOOTHROT_INVALID_ARG;
+  if (Xq == nullptr || Wq == nullptr) return SMOOTHROT_INVALID_ARG;
+  if (!aligned16(Xq) || !aligned16(Wq)) return SMOOTHROT_BAD_ALIGNMENT;
+  if (Y != nullptr) {
+    if (dx == nullptr || dw == nullptr || ldy < N) return SMOOTHROT_INVALID_ARG;
+    if (!aligned16(Y) || ldy % 8 != 0 || !aligned16(dw)) return SMOOTHROT_BAD_ALIGNMENT;
+  } else {
+    if (acc_out == nullptr) return SMOOTHROT_INVALID_ARG;
+    if (!aligned16(acc_out)) return SMOOTHROT_BAD_ALIGNMENT;
+  }
+  const Plan pl = make_plan(M, N, K);
+  const size_t need = pl.splits > 1 ? size_t(pl.splits) * size_t(M) * size_t(N) * sizeof(int32_t) : 0;
+  if (need > 0 && (workspace == nullptr || workspace_bytes < need)) return SMOOTHROT_WORKSPACE_TOO_SMALL;
+  if (need > 0 && !aligned16(workspace)) return SMOOTHROT_BAD_ALIGNMENT;
+
+  Params p{};
+  p.swapped = pl.swapped ? 1 : 0;
+  const uint8_t* a_ptr = pl.swapped ? Wq : Xq;
+  const uint8_t* b_ptr = pl.swapped ? Xq : Wq;
+  p.rows_a = int(pl.swapped ? N : M);
+  p.rows_b = int(pl.swapped ? M : N);
+  p.tiles_a = (p.rows_a + kBM - 1) / kBM;
+  p.tiles_b = (p.rows_b + pl.bn - 1) / pl.bn;
+  p.kblocks = int(K / kWideRow);
+  p.splits = pl.splits;
+  p.M = int(M);
+  p.N = int(N);
+  p.dx = dx;
+  p.dw = dw;
+  p.ldy = ldy;
+  if (pl.splits > 1) {
+    p.Y = nullptr;
+    p.acc_out = static_cast<int32_t*>(workspace);
+  } else {
+    p.Y = Y;
+    p.acc_out = Y ? nullptr : acc_out;
+  }
+  CUtensorMap ma, mb;
+  if (!make_map(&ma, a_ptr, p.rows_a, K, kBM) || !make_map(&mb, b_ptr, p.rows_b, K, pl.bn))
+    return SMOOTHROT_CUDA_ERROR;
+  int rc;
+  switch (pl.bn) {
+    case 256: rc = launch_tile<256>(ma, mb, p, st); break;
+    case 128: rc = launch_tile<128>(ma, mb, p, st); break;
+    case 64: rc = launch_tile<64>(ma, mb, p, st); break;
+    case 32: rc = launch_tile<32>(ma, mb, p, st); break;
+    default: rc = launch_tile<16>(ma, mb, p, st); break;
+  }
+  if (rc != SMOOTHROT_OK) return rc;
+  if (pl.splits > 1) {
+    const int64_t total = M * N;
+    const int threads = 256;
+    splitk_reduce_kernel<<<unsigned((total + threads - 1) / threads), threads, 0, st>>>(
+        static_cast<const int32_t*>(workspace), pl.splits, int(M), int(N), dx, dw, Y, ldy, acc_out);
+    count_launch();
+    rc = launch_status();
+  }
+  return rc;
+}
+
+}  // namespace gemm
+}  // namespace smoothrot
+
+extern "C" {
+
+size_t smoothrot_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+  if (M <= 0 || N <= 0 || K <= 0 || K % smoothrot::gemm::kWideRow != 0) return 0;
+  const smoothrot::gemm::Plan pl = smoothrot::gemm::make_plan(M, N, K);
+  return pl.splits > 1 ? size_t(pl.splits) * size_t(M) * size_t(N) * sizeof(int32_t) : 0;
+}
+
+int smoothrot_linear(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq, const float* dw,
+                     int64_t N, int64_t K, void* Y_f16, int64_t ldy, void* workspace, size_t workspace_bytes,
+                     void* stream) {
+  if (M > 0 && N > 0 && Y_f16 == nullptr) return SMOOTHROT_INVALID_ARG;
+  return smoothrot::gemm::run(Xq, dx, M, Wq, dw, N, K, static_cast<__half*>(Y_f16), ldy, nullptr, workspace,
+                              workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+int smoothrot_debug_gemm_i32(const uint8_t* Xq, int64_t M, const uint8_t* Wq, int64_t N, int64_t K,
+                             int32_t* acc, void* workspace, size_t workspace_bytes, void* stream) {
+  if (M > 0 && N > 0 && acc == nullptr) return SMOOTHROT_INVALID_ARG;
+  return smoothrot::gemm::run(Xq, nullptr, M, Wq, nullptr, N, K, nullptr, 0, acc, workspace, workspace_bytes,
+                              static_cast<cudaStream_t>(stream));
+}
+
+int smoothrot_device_status(int* status_host, int clear) {
+  if (status_host == nullptr) return SMOOTHROT_INVALID_ARG;
+  int v = 0;
+  if (cudaMemcpyFromSymbol(&v, smoothrot::gemm::g_device_status, sizeof(int)) != cudaSuccess)
+    return SMOOTHROT_CUDA_ERROR;
+  *status_host = v;
+  if (clear && v != 0) {
+    const int zero = 0;
+    if (cudaMemcpyToSymbol(smoothrot::gemm::g_device_status, &zero, sizeof(int)) != cudaSuccess)
+      return SMOOTHROT_CUDA_ERROR;
+  }
+  return SMOOTHROT_OK;
+}
+
+}  // extern "C"

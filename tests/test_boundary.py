@@ -1,0 +1,83 @@
+"""The C-ABI boundary without a GPU: the library loads, exports every symbol
+the header declares, and rejects bad arguments before touching the device."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "smoothrot.h")
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2506_05413_b200 import build, binding
+    build.build()
+    return binding.load()
+
+
+def _declared():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(smoothrot_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported_and_bound(lib):
+    from paper_2506_05413_b200 import binding
+    names = _declared()
+    assert "smoothrot_quant_act" in names and "smoothrot_linear" in names and len(names) >= 11
+    for n in names:
+        assert hasattr(lib, n), n
+        assert n in binding.SIGNATURES, f"{n} has no ctypes signature"
+    assert sorted(binding.SIGNATURES) == names
+
+
+def test_status_strings(lib):
+    from paper_2506_05413_b200 import binding
+    assert binding.status_string(0) == "ok"
+    texts = {binding.status_string(c) for c in range(-6, 1)}
+    assert len(texts) == 7 and binding.status_string(-99) == "unknown status"
+
+
+def test_host_side_rejections(lib):
+    dummy = ctypes.c_void_p(0x1000)   # never dereferenced: each call fails validation first
+    odd = ctypes.c_void_p(0x1008)
+    q = lib.smoothrot_quant_act
+    assert q(dummy, 4, 100, 104, None, 0.9, dummy, dummy, None) == -2        # unsupported K
+    assert q(dummy, 4, 64, 64, None, 0.9, dummy, dummy, None) == -2          # 2^6 too small
+    assert q(dummy, 4, 28 * 1024, 28 * 1024, None, 0.9, dummy, dummy, None) == -2
+    assert q(dummy, -1, 128, 128, None, 0.9, dummy, dummy, None) == -1       # negative rows
+    assert q(None, 4, 128, 128, None, 0.9, dummy, dummy, None) == -1         # null input
+    assert q(dummy, 4, 128, 64, None, 0.9, dummy, dummy, None) == -1         # ld < K
+    assert q(odd, 4, 128, 128, None, 0.9, dummy, dummy, None) == -3          # misaligned
+    assert q(dummy, 4, 128, 132, None, 0.9, dummy, dummy, None) == -3        # ld not multiple of 8
+    assert q(dummy, 4, 128, 128, None, 0.0, dummy, dummy, None) == -1        # clip out of range
+    assert q(dummy, 4, 128, 128, None, 1.5, dummy, dummy, None) == -1
+    assert q(dummy, 0, 128, 128, None, 0.9, None, None, None) == 0           # empty input is fine
+    assert lib.smoothrot_fuse_weights(dummy, 4, 96, 96, None, 1.0, dummy, dummy, None) == -2
+    lin = lib.smoothrot_linear
+    assert lin(dummy, dummy, 4, dummy, dummy, 8, 100, dummy, 8, None, 0, None) == -2   # K % 128
+    assert lin(dummy, dummy, 4, dummy, dummy, 12, 128, dummy, 16, None, 0, None) == -1  # N % 8
+    assert lin(dummy, dummy, 4, dummy, dummy, 8, 128, dummy, 4, None, 0, None) == -1   # ldy < N
+    assert lin(odd, dummy, 4, dummy, dummy, 8, 128, dummy, 8, None, 0, None) == -3
+    assert lin(dummy, dummy, 0, dummy, dummy, 8, 128, dummy, 8, None, 0, None) == 0
+    # a shape that splits K needs a workspace
+    need = lib.smoothrot_workspace_bytes(4, 1024, 4096)
+    assert need > 0 and need % (4 * 1024 * 4) == 0
+    assert lin(dummy, dummy, 4, dummy, dummy, 1024, 4096, dummy, 1024, None, 0, None) == -4
+    assert lin(dummy, dummy, 4, dummy, dummy, 1024, 4096, dummy, 1024, dummy, need - 1, None) == -4
+    assert lib.smoothrot_workspace_bytes(2048, 6144, 4096) == 0
+    cal = lib.smoothrot_calibrate
+    assert cal(dummy, 4, 128, 128, None, 0, 0, 0.5, 1, dummy, dummy, None, None, None, None) == -1  # finalize, no W
+    assert cal(dummy, 4, 128, 128, dummy, 4, 128, 1.5, 1, dummy, dummy, None, None, None, None) == -1  # alpha
+    assert cal(dummy, 4, 128, 128, None, 0, 0, 0.5, 0, None, None, None, None, None, None) == -1
+    assert lib.smoothrot_paley28(None) == -1
+    assert lib.smoothrot_device_status(None, 0) == -1
+
+
+def test_library_paley_table_equals_oracle_table(lib):
+    import numpy as np
+    from oracle import smoothrot_oracle as orc
+    from paper_2506_05413_b200 import binding
+    assert np.array_equal(np.array(binding.paley28(), dtype=np.int8), orc.paley28())

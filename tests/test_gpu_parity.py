@@ -1,0 +1,226 @@
+"""GPU-vs-oracle parity, call by call, through the C-ABI binding.
+
+Tolerances (written here once):
+  * rotation (debug export): per row ||y_gpu - y_oracle||_inf / ||y_oracle||_inf <= 1e-5
+  * step sizes and smoothing scales: <= 1e-6 relative
+  * packed codes: at most 1e-4 of the codes differ from the oracle's and every
+    difference is +-1 (rounding ties moved by fp32 summation order)
+  * int32 accumulators: bit-exact, and identical from run to run
+  * fp16 outputs: per row <= 2e-3 relative to the row maximum of the oracle fed the GPU's codes
+"""
+import numpy as np
+import pytest
+
+from oracle import smoothrot_oracle as orc
+from paper_2506_05413_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+TOL_ROT = 1e-5
+TOL_SCALE = 1e-6
+TOL_CODES = 1e-4
+TOL_OUT = 2e-3
+
+
+@pytest.fixture(scope="module")
+def gu():
+    from paper_2506_05413_b200 import build
+    build.build()
+    import gpu_util
+    return gpu_util
+
+
+def _acts(seed, M, K, gain=1000.0):
+    rng = np.random.default_rng(seed)
+    tok = np.arange(0, M, 17)
+    ch = np.sort(rng.choice(K, size=3, replace=False))
+    return synth.activations(rng, M, K, law="normal", outlier_channels=ch, outlier_gain=gain,
+                             outlier_tokens=tok)
+
+
+def _pre(seed, K):
+    rng = np.random.default_rng(seed)
+    return (rng.uniform(0.02, 8.0, K) * (rng.integers(0, 2, K) * 2 - 1)).astype(np.float32)
+
+
+# ------------------------------------------------------------------ rotation
+@pytest.mark.parametrize("K,M", [(128, 64), (256, 5), (512, 33), (1024, 7), (2048, 3), (4096, 37),
+                                 (4096, 4), (8192, 2), (28 * 8, 9), (28 * 64, 5), (14336, 11)])
+@pytest.mark.parametrize("use_pre", [False, True])
+def test_rotation_matches_oracle(gu, K, M, use_pre):
+    X = _acts(K + M, M, K)
+    pre = _pre(K, K) if use_pre else None
+    got = gu.gpu_hadamard(X, pre)
+    want = orc.rotate(X, pre, K)
+    assert gu.rowwise_rel(got, want) <= TOL_ROT
+
+
+def test_rotation_closed_forms_on_gpu(gu):
+    for K in (128, 4096, 14336):
+        X = np.zeros((2, K), np.float16)
+        X[0, 5] = 3.0
+        X[1, :] = 0.5
+        got = gu.gpu_hadamard(X, None)
+        assert np.allclose(np.abs(got[0]), 3.0 / np.sqrt(K), rtol=1e-6)
+        if K != 14336:
+            want = np.zeros(K); want[0] = 0.5 * np.sqrt(K)
+            assert np.allclose(got[1], want, atol=1e-4)
+
+
+def test_rotation_with_row_stride(gu):
+    import torch
+    from paper_2506_05413_b200 import binding as sr
+    K, M = 4096, 6
+    X = _acts(3, M, K)
+    big = torch.zeros((M, K + 64), dtype=torch.float16, device=gu.DEV)
+    big[:, :K] = gu.dev(X)
+    Y = torch.empty((M, K), dtype=torch.float32, device=gu.DEV)
+    sr.debug_hadamard(big[:, :K], None, Y)
+    torch.cuda.synchronize()
+    assert gu.rowwise_rel(Y.cpu().numpy(), orc.rotate(X, None, K)) <= TOL_ROT
+
+
+# ------------------------------------------------------- quantize + pack
+@pytest.mark.parametrize("K,M", [(128, 64), (512, 21), (4096, 301), (4096, 1), (8192, 3), (28 * 16, 10), (14336, 19)])
+@pytest.mark.parametrize("which", ["act", "weight"])
+def test_quantized_codes_match_oracle(gu, K, M, which):
+    from paper_2506_05413_b200 import binding as sr
+    X = _acts(7 * K + M, M, K) if which == "act" else \
+        (np.random.default_rng(K).standard_normal((M, K)) * 0.02).astype(np.float16)
+    pre = _pre(K + 1, K)
+    clip = 0.9 if which == "act" else 1.0
+    fn = sr.quant_act if which == "act" else sr.fuse_weights
+    q, step = gu.gpu_quantize(fn, X, pre, clip)
+    ofn = orc.quant_act if which == "act" else orc.fuse_weights
+    q_ref, step_ref, _ = ofn(X, pre, K, clip)
+    assert np.abs(step / step_ref - 1).max() <= TOL_SCALE
+    frac, worst = gu.code_mismatch(q, q_ref)
+    assert worst <= 1 and frac <= max(TOL_CODES, 1.5 / q.size / 2)
+    codes = orc.unpack_codes(q)
+    assert codes.min() >= -8 and codes.max() <= 7
+
+
+def test_quantizer_edge_rows(gu):
+    from paper_2506_05413_b200 import binding as sr
+    for K in (128, 4096, 14336):
+        X = np.zeros((3, K), np.float16)
+        X[1, 9] = -2.0                     # unit vector: every |x^| equal -> codes +7 / -8
+        X[2, :] = 65504.0                  # largest fp16 everywhere
+        q, step = gu.gpu_quantize(sr.quant_act, X, None, 0.9)
+        codes = orc.unpack_codes(q)
+        assert step[0] == np.float32(1.0) and np.all(codes[0] == 0)
+        assert set(np.unique(codes[1])) <= {7, -8}
+        H = orc.hadamard_matrix(K)
+        assert np.array_equal(codes[1] == -8, H[9] > 0)      # x^ = -2 H[9] / sqrt(K)
+        assert np.all(np.isfinite(step))
+        q_ref, step_ref, _ = orc.quant_act(X, None, K, 0.9)
+        assert np.abs(step / step_ref - 1).max() <= TOL_SCALE
+
+
+# ------------------------------------------------------------- calibration
+@pytest.mark.parametrize("K,T,N,batches", [(128, 128, 256, 1), (4096, 300, 77, 3), (14336, 65, 130, 2)])
+def test_calibration_matches_oracle(gu, K, T, N, batches):
+    rng = np.random.default_rng(K + T)
+    Xc = _acts(K, T, K)
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float16)
+    W[:, 3] = 0                                            # dead weight channel -> eps guard
+    d = synth.sign_vector(rng, K)
+    for alpha in (0.5, 0.45, 0.0, 1.0):
+        amax, s, pre_w, pre_x = gu.gpu_calibrate(Xc, W, alpha, d, batches)
+        amax_ref, s_ref = orc.calibrate(Xc, W, alpha)
+        assert np.array_equal(amax, amax_ref)
+        assert np.abs(s / s_ref - 1).max() <= TOL_SCALE
+        assert np.array_equal(pre_w, s * d)
+        assert np.array_equal(pre_x, (d.astype(np.float64) / s.astype(np.float64)).astype(np.float32))
+
+
+# --------------------------------------------------------------------- GEMM
+GEMM_SHAPES = [
+    (64, 256, 128),      # config 0
+    (1, 1024, 4096),     # decode, split K
+    (4, 4096, 4096),
+    (16, 136, 512),
+    (17, 64, 256),       # 32-wide token tile
+    (33, 72, 384),       # 64-wide token tile
+    (100, 264, 256),     # 128-wide token tile, swapped
+    (128, 64, 128),      # prefill, BN = 64
+    (130, 136, 640),     # BN = 128, ragged both ways
+    (300, 520, 1152),    # BN = 256, several tiles and a ragged tail
+    (257, 8, 128),
+    (512, 1024, 14336),  # long K
+]
+
+
+@pytest.mark.parametrize("M,N,K", GEMM_SHAPES)
+def test_gemm_accumulators_bit_exact(gu, M, N, K):
+    xq = synth.random_codes(M * 31 + K, M, K)
+    wq = synth.random_codes(N * 17 + K + 1, N, K)
+    got = gu.gpu_gemm_i32(orc.pack_codes(xq), orc.pack_codes(wq))
+    want = orc.gemm_i32(xq, wq)
+    assert np.array_equal(got, want)
+    again = gu.gpu_gemm_i32(orc.pack_codes(xq), orc.pack_codes(wq))
+    assert np.array_equal(got, again)
+
+
+def test_gemm_extreme_codes(gu):
+    K = 14336
+    xq = np.full((130, K), -8, np.int8)
+    wq = np.full((264, K), -8, np.int8)
+    wq[1::2] = 7
+    got = gu.gpu_gemm_i32(orc.pack_codes(xq), orc.pack_codes(wq))
+    assert np.all(got[:, 0::2] == 64 * K) and np.all(got[:, 1::2] == -56 * K)
+
+
+@pytest.mark.parametrize("M,N,K", [(64, 256, 128), (3, 1024, 4096), (200, 264, 512), (130, 520, 4096)])
+def test_linear_output_matches_oracle_on_gpu_codes(gu, M, N, K):
+    rng = np.random.default_rng(M + N + K)
+    xq = orc.pack_codes(synth.random_codes(M, M, K))
+    wq = orc.pack_codes(synth.random_codes(N + 1, N, K))
+    dx = rng.uniform(0.01, 0.3, M).astype(np.float32)
+    dw = rng.uniform(1e-4, 4e-3, N).astype(np.float32)
+    got = gu.gpu_linear(xq, dx, wq, dw)
+    want = orc.linear(xq, dx, wq, dw)
+    assert np.isfinite(got.astype(np.float32)).all()
+    assert gu.rowwise_rel(got, want) <= TOL_OUT
+
+
+# ------------------------------------------------------------- whole layer
+def _layer_on_gpu(gu, case):
+    from paper_2506_05413_b200 import binding as sr
+    amax, s, pre_w, pre_x = gu.gpu_calibrate(case.X_calib, case.W, case.alpha, case.d)
+    wq, dw = gu.gpu_quantize(sr.fuse_weights, case.W, pre_w, case.clip_w)
+    xq, dx = gu.gpu_quantize(sr.quant_act, case.X, pre_x, case.clip_a)
+    Y = gu.gpu_linear(xq, dx, wq, dw)
+    return dict(amax=amax, s=s, pre_w=pre_w, pre_x=pre_x, wq=wq, dw=dw, xq=xq, dx=dx, Y=Y)
+
+
+def _check_layer(gu, case, g):
+    K = case.K
+    amax_ref, s_ref = orc.calibrate(case.X_calib, case.W, case.alpha)
+    assert np.array_equal(g["amax"], amax_ref)
+    assert np.abs(g["s"] / s_ref - 1).max() <= TOL_SCALE
+    # staged: each oracle stage is fed the GPU's upstream outputs
+    wq_ref, dw_ref, _ = orc.fuse_weights(case.W, g["pre_w"], K, case.clip_w)
+    xq_ref, dx_ref, _ = orc.quant_act(case.X, g["pre_x"], K, case.clip_a)
+    assert np.abs(g["dw"] / dw_ref - 1).max() <= TOL_SCALE
+    assert np.abs(g["dx"] / dx_ref - 1).max() <= TOL_SCALE
+    for got, ref in ((g["wq"], wq_ref), (g["xq"], xq_ref)):
+        frac, worst = gu.code_mismatch(got, ref)
+        assert worst <= 1 and frac <= TOL_CODES
+    Y_ref = orc.linear(g["xq"], g["dx"], g["wq"], g["dw"])
+    assert gu.rowwise_rel(g["Y"], Y_ref) <= TOL_OUT
+
+
+def test_config0_whole_layer(gu):
+    case = synth.config0()
+    g = _layer_on_gpu(gu, case)
+    _check_layer(gu, case, g)
+    Yfp = case.X.astype(np.float64) @ case.W.astype(np.float64).T
+    err = np.linalg.norm(g["Y"].astype(np.float64) - Yfp) / np.linalg.norm(Yfp)
+    assert err < 0.25
+
+
+@pytest.mark.parametrize("maker,M,N", [(synth.config1, 160, 264), (synth.config2, 130, 136), (synth.config3, 40, 520)])
+def test_reduced_configs_whole_layer(gu, maker, M, N):
+    case = maker(M=M, N=N)
+    _check_layer(gu, case, _layer_on_gpu(gu, case))
