@@ -1,0 +1,400 @@
+#!/usr/bin/env python
+"""Benchmark of the SmoothRot W4A4 linear layer on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg1|cfg2|cfg3]
+    python bench.py --impl reference ...        # the CPU oracle on the host cores
+
+One "step" is one pass of the whole path over one batch of seeded synthetic
+input: calibrate (per-channel absmax -> scales), fuse_weights (scale, rotate,
+quantize, pack W), quant_act (Hadamard + per-token INT4 quantize + pack X) and
+linear (INT4 x INT4 GEMM + dequant to fp16).  The headline value is the layer's
+2*M*N*K integer operations divided by the time of the whole step.
+
+The device-timed region keeps every input resident in HBM; between steps the
+loop rotates through several distinct buffer sets whose total size exceeds
+twice the L2 capacity, so no step finds its inputs in L2.  The end-to-end
+figure starts from pinned host buffers and ends with the output back on the
+host, with the copies inside the timed region.
+
+Prints exactly one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2506_05413_b200 import synth  # noqa: E402
+
+L2_BYTES = 126 * 1024 * 1024
+NOMINAL_INT8_TOPS = 4500.0
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+METRIC = "w4a4_smoothrot_linear_tops"
+UNIT = "TOPS"
+
+WORKLOADS = {
+    "cfg0": (synth.config0, "configs[0]: tiny layer, X [64 x 128], W [256 x 128]"),
+    "cfg1": (synth.config1, "configs[1]: LLaMA-3.1-8B-shaped fused QKV, X [2048 x 4096], W [6144 x 4096]"),
+    "cfg2": (synth.config2, "configs[2]: down_proj with online Hadamard, X [2048 x 14336], W [4096 x 14336]"),
+    "cfg3": (synth.config3, "configs[3]: fused gate/up, X [8192 x 4096], W [28672 x 4096]"),
+}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16=float(p["bf16_tflops"]),
+                    bf16_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=FALLBACK_HBM_GBS, bf16=FALLBACK_BF16_TFLOPS, bf16_sustained=1400.0, source="fallback")
+
+
+def layer_ops(M, N, K):
+    return 2.0 * M * N * K
+
+
+def algorithmic_bytes(M, N, K, T):
+    """Bytes each call must move at least once (fp16 in, packed codes out, fp32 scales)."""
+    return {
+        "calibrate": 2.0 * T * K + 2.0 * N * K + 4.0 * K * 5,
+        "fuse_weights": 2.0 * N * K + 0.5 * N * K + 4.0 * N + 4.0 * K,
+        "quant_act": 2.0 * M * K + 0.5 * M * K + 4.0 * M + 4.0 * K,
+        "linear": 0.5 * M * K + 0.5 * N * K + 2.0 * M * N + 4.0 * (M + N),
+    }
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.lines = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.QUERY}",
+                 "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._pump, daemon=True)
+        self.thread.start()
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0])); smax.append(float(parts[1])); power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, flag in zip(names, parts[4:8]):
+                if flag.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(smax)),
+                "power_w_max": float(max(power)), "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------
+# The CPU oracle arm (also the cpu_baseline leg of the GPU arm)
+# ---------------------------------------------------------------------------
+def oracle_step(case, Ms, Ns):
+    """One pass of the whole path by the oracle on the first Ms tokens and Ns
+    output channels of the workload (full K, full calibration set); returns seconds."""
+    from oracle import smoothrot_oracle as orc
+    t0 = time.perf_counter()
+    orc.smoothrot_layer(case.X[:Ms], case.X_calib, case.W[:Ns], case.d, case.alpha, case.clip_a, case.clip_w)
+    return time.perf_counter() - t0
+
+
+def oracle_sample_shape(case):
+    """A bounded sample of the workload: the whole layer if its GEMM has at most
+    6e10 multiply-adds (a few seconds for the plain C loop), else the leading
+    tokens / output channels, halved in turn until it does."""
+    Ms, Ns = case.M, case.N
+    while float(Ms) * Ns * case.K > 6e10:
+        if Ms >= Ns and Ms > 1:
+            Ms //= 2
+        else:
+            Ns = max(8, Ns // 2)
+    return Ms, Ns
+
+
+def oracle_threads():
+    from oracle import smoothrot_oracle as orc
+    return orc.gemm_threads()
+
+
+def run_reference(args, case, desc):
+    Ms, Ns = oracle_sample_shape(case)
+    for _ in range(min(args.warmup, 1)):
+        oracle_step(case, Ms, Ns)
+    steps = max(1, min(args.steps, 3))
+    t = [oracle_step(case, Ms, Ns) for _ in range(steps)]
+    sec = float(np.mean(t))
+    value = layer_ops(Ms, Ns, case.K) / sec / 1e12
+    sample = f"first {Ms} tokens x first {Ns} output channels, full K = {case.K}, whole path per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int4", "data": "synthetic",
+        "config": {"workload": desc, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------
+# The GPU arm
+# ---------------------------------------------------------------------------
+class DeviceSet:
+    """One resident copy of a layer's inputs and outputs."""
+
+    def __init__(self, torch, sr, case, dev):
+        t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+        M, N, K = case.M, case.N, case.K
+        self.X, self.Xc, self.W, self.d = t(case.X), t(case.X_calib), t(case.W), t(case.d)
+        f32 = lambda n: torch.empty(n, dtype=torch.float32, device=dev)
+        self.amax, self.s, self.pre_w, self.pre_x = f32(K), f32(K), f32(K), f32(K)
+        self.wq = torch.empty((N, K // 2), dtype=torch.uint8, device=dev)
+        self.xq = torch.empty((M, K // 2), dtype=torch.uint8, device=dev)
+        self.dw, self.dx = f32(N), f32(M)
+        self.Y = torch.empty((M, N), dtype=torch.float16, device=dev)
+        need = sr.workspace_bytes(M, N, K)
+        self.ws = torch.empty(need, dtype=torch.uint8, device=dev) if need else None
+
+    def nbytes(self):
+        tensors = (self.X, self.Xc, self.W, self.wq, self.xq, self.Y)
+        return sum(x.numel() * x.element_size() for x in tensors)
+
+
+CALLS = ("calibrate", "fuse_weights", "quant_act", "linear")
+
+
+def gpu_step(sr, case, ds, events=None):
+    """The whole path on one buffer set.  With `events`, each call is bracketed
+    by a pair of CUDA events on the launching stream."""
+    def mark(i, which):
+        if events is not None:
+            events[i][which].record()
+    ds.amax.zero_()
+    mark(0, 0)
+    sr.calibrate(ds.Xc, ds.amax, W=ds.W, alpha=case.alpha, s_out=ds.s, d=ds.d,
+                 pre_w_out=ds.pre_w, pre_x_out=ds.pre_x)
+    mark(0, 1); mark(1, 0)
+    sr.fuse_weights(ds.W, ds.pre_w, case.clip_w, ds.wq, ds.dw)
+    mark(1, 1); mark(2, 0)
+    sr.quant_act(ds.X, ds.pre_x, case.clip_a, ds.xq, ds.dx)
+    mark(2, 1); mark(3, 0)
+    sr.linear(ds.xq, ds.dx, ds.wq, ds.dw, ds.Y, ds.ws)
+    mark(3, 1)
+
+
+def run_gpu(args, case, desc):
+    import torch
+    from paper_2506_05413_b200 import binding as sr
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    sr.load()
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    M, N, K, T = case.M, case.N, case.K, case.X_calib.shape[0]
+    first = DeviceSet(torch, sr, case, dev)
+    n_sets = max(2, int(np.ceil(2.2 * L2_BYTES / first.nbytes())))
+    sets = [first]
+    for i in range(1, n_sets):
+        ds = DeviceSet(torch, sr, case, dev)
+        sets.append(ds)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        gpu_step(sr, case, sets[i % n_sets])
+    torch.cuda.synchronize()
+    assert sr.device_status() == 0, "a device-side wait timed out during warm-up"
+
+    # ---- device-timed region: K steps, per-call events inside -------------------
+    ev = [[[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in CALLS] for _ in range(args.steps)]
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = sr.launch_count()
+    barrier()
+    start.record()
+    for i in range(args.steps):
+        gpu_step(sr, case, sets[i % n_sets], ev[i])
+    stop.record()
+    barrier()
+    launches = sr.launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = start.elapsed_time(stop)
+    if dist is not None:
+        tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    ms_per_step = total_ms / args.steps
+    call_ms = {name: float(np.mean([ev[i][c][0].elapsed_time(ev[i][c][1]) for i in range(args.steps)]))
+               for c, name in enumerate(CALLS)}
+    assert sr.device_status() == 0, "a device-side wait timed out"
+
+    # ---- end to end: pinned host inputs -> device -> path -> output on the host ----
+    ds = sets[0]
+    host_in = [torch.from_numpy(np.ascontiguousarray(a)).pin_memory() for a in (case.X, case.X_calib, case.W, case.d)]
+    dev_in = [ds.X, ds.Xc, ds.W, ds.d]
+    host_Y = torch.empty((M, N), dtype=torch.float16).pin_memory()
+    h2d = sum(h.numel() * h.element_size() for h in host_in)
+    d2h = host_Y.numel() * host_Y.element_size()
+
+    def e2e_step():
+        for h, d_ in zip(host_in, dev_in):
+            d_.copy_(h, non_blocking=True)
+        gpu_step(sr, case, ds)
+        host_Y.copy_(ds.Y, non_blocking=True)
+        torch.cuda.synchronize()
+
+    for _ in range(3):
+        e2e_step()
+    e2e_steps = max(3, min(args.steps, 20))
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    barrier()
+    e2e_sec = (time.perf_counter() - t0) / e2e_steps
+    if dist is not None:
+        tt = torch.tensor([e2e_sec], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_sec = float(tt.item())
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    ops = layer_ops(M, N, K)
+    peaks = measured_peaks()
+    int8_peak = peaks["bf16"] * (NOMINAL_INT8_TOPS / NOMINAL_BF16_TFLOPS)
+    abytes = algorithmic_bytes(M, N, K, T)
+    dominant = max(call_ms, key=call_ms.get)
+    if dominant == "linear":
+        achieved = ops / (call_ms["linear"] * 1e-3) / 1e12
+        roofline = {"kernel": "w4a4_gemm_kernel (smoothrot_linear)", "bound": "tensor", "achieved": achieved,
+                    "peak": int8_peak, "unit": "TOP/s", "frac": achieved / int8_peak, "traffic": None,
+                    "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16']} TFLOP/s x 2 (nominal int8:bf16 ratio)",
+                    "frac_of_nominal_4500": achieved / NOMINAL_INT8_TOPS}
+    else:
+        achieved = abytes[dominant] / (call_ms[dominant] * 1e-3) / 1e9
+        roofline = {"kernel": dominant, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                    "peak_source": f"{peaks['source']} copy bandwidth"}
+    per_call = {}
+    for name in CALLS:
+        sec = call_ms[name] * 1e-3
+        per_call[name] = {"ms": call_ms[name], "GB/s": abytes[name] / sec / 1e9,
+                          "frac_hbm": abytes[name] / sec / 1e9 / peaks["hbm_gbs"]}
+    per_call["linear"]["TOPS"] = ops / (call_ms["linear"] * 1e-3) / 1e12
+    per_call["linear"]["frac_int8_peak"] = per_call["linear"]["TOPS"] / int8_peak
+
+    # ---- the oracle on this machine's host cores, bounded sample ----------------------
+    Ms, Ns = oracle_sample_shape(case)
+    cpu_sec = oracle_step(case, Ms, Ns)
+    cpu_value = layer_ops(Ms, Ns, K) / cpu_sec / 1e12
+    sample = f"first {Ms} tokens x first {Ns} output channels, full K = {K}, whole path once ({cpu_sec:.1f} s)"
+
+    line = {
+        "metric": METRIC, "value": world * ops / (ms_per_step * 1e-3) / 1e12, "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int4", "data": "synthetic",
+        "config": {"workload": desc, "M": M, "N": N, "K": K, "calib_tokens": T, "alpha": case.alpha,
+                   "step": "calibrate + fuse_weights + quant_act + linear",
+                   "l2": f"inputs rotate through {n_sets} buffer sets ({n_sets * first.nbytes() / 2**20:.0f} MiB > 2 x L2)",
+                   "parallelism": "replicas only" if world > 1 else "1 GPU"},
+        "clocks": clocks,
+        "e2e": {"value": world * ops / e2e_sec / 1e12, "unit": UNIT, "ms_per_step": e2e_sec * 1e3,
+                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+        "cpu_baseline": {"value": cpu_value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+                         "sample": sample},
+        "per_call": per_call,
+        "online_only": {"ms": call_ms["quant_act"] + call_ms["linear"],
+                        "TOPS": ops / ((call_ms["quant_act"] + call_ms["linear"]) * 1e-3) / 1e12},
+    }
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
+    ap.add_argument("--workload", choices=sorted(WORKLOADS), default="cfg1")
+    args = ap.parse_args()
+    maker, desc = WORKLOADS[args.workload]
+    rank = int(os.environ.get("RANK", "0"))
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        run_reference(args, maker(), desc)
+        return
+    run_gpu(args, maker(), desc)
+
+
+if __name__ == "__main__":
+    main()
