@@ -55,7 +55,8 @@ typedef enum {
   SMOOTHROT_BAD_ALIGNMENT = -3,       /* pointer or leading dimension misaligned */
   SMOOTHROT_WORKSPACE_TOO_SMALL = -4, /* see smoothrot_workspace_bytes */
   SMOOTHROT_CUDA_ERROR = -5,          /* a CUDA runtime / driver call failed */
-  SMOOTHROT_DEVICE_TIMEOUT = -6       /* a bounded wait inside a kernel ran out */
+  SMOOTHROT_DEVICE_TIMEOUT = -6,      /* a bounded wait inside a kernel ran out */
+  SMOOTHROT_STATIC_SCRATCH_EXCEEDED = -7 /* shape needs more than SMOOTHROT_STATIC_SCRATCH_BYTES */
 } smoothrot_status;
 
 /* Host. Text for a status code; never NULL. */
@@ -130,6 +131,43 @@ int smoothrot_linear(const uint8_t* Xq, const float* dx, int64_t M,
                      const uint8_t* Wq, const float* dw, int64_t N, int64_t K,
                      void* Y_f16, int64_t ldy,
                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * smoothrot_linear without a caller-provided workspace.  (An addition of this
+ * library; the paper has no counterpart.)
+ *
+ * Who needs it: code that must run the layer but is not in a position to
+ * obtain device memory for the split-K scratch.  Typical cases are a plug-in
+ * inside a serving process whose host application handed out all device
+ * memory at start-up and forbids cudaMalloc afterwards, a component that is
+ * only ever given the input and output buffers of the layer, or a process in
+ * which cudaMalloc would fail because another allocator has already reserved
+ * the whole device.  For such callers the scratch lives inside the library: a
+ * fixed array of SMOOTHROT_STATIC_SCRATCH_BYTES in device memory that belongs
+ * to the loaded module.  Every GPU on which the library is used keeps that
+ * many bytes occupied until the process exits, whether or not this entry
+ * point is ever called there.
+ *
+ * Same arguments, results and error behaviour as smoothrot_linear, minus the
+ * workspace pair.  The call itself allocates and frees nothing.  Shapes whose
+ * smoothrot_workspace_bytes(M, N, K) exceeds SMOOTHROT_STATIC_SCRATCH_BYTES
+ * are refused with SMOOTHROT_STATIC_SCRATCH_EXCEEDED and nothing is enqueued
+ * (use smoothrot_linear with your own workspace for those).
+ *
+ * The first call on each device looks up the array's device address
+ * (cudaGetSymbolAddress, with that device current) and remembers it; make that
+ * first call before starting any stream capture on the device.
+ *
+ * There is ONE array per device, shared by every call: two calls whose work
+ * may overlap on the GPU (different streams, or several host threads) race on
+ * it and produce garbage.  Calls on one stream are safe.  The array keeps
+ * whatever the previous call left; this entry point never depends on those
+ * contents, because each call overwrites every partial sum it later reads.
+ */
+#define SMOOTHROT_STATIC_SCRATCH_BYTES (8u * 1024u * 1024u)
+int smoothrot_linear_static_scratch(const uint8_t* Xq, const float* dx, int64_t M,
+                                    const uint8_t* Wq, const float* dw, int64_t N, int64_t K,
+                                    void* Y_f16, int64_t ldy, void* stream);
 
 /* Host. Scratch bytes smoothrot_linear / smoothrot_debug_gemm_i32 need for
  * this shape (0 for shapes that need none). */

@@ -25,6 +25,7 @@ SIGNATURES = {
     "smoothrot_fuse_weights": (_int, [_vp, _i64, _i64, _i64, _vp, _f32, _vp, _vp, _vp]),
     "smoothrot_quant_act": (_int, [_vp, _i64, _i64, _i64, _vp, _f32, _vp, _vp, _vp]),
     "smoothrot_linear": (_int, [_vp, _vp, _i64, _vp, _vp, _i64, _i64, _vp, _i64, _vp, _sz, _vp]),
+    "smoothrot_linear_static_scratch": (_int, [_vp, _vp, _i64, _vp, _vp, _i64, _i64, _vp, _i64, _vp]),
     "smoothrot_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "smoothrot_debug_hadamard": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp]),
     "smoothrot_debug_gemm_i32": (_int, [_vp, _i64, _vp, _i64, _i64, _vp, _vp, _sz, _vp]),
@@ -163,6 +164,25 @@ def linear(Xq, dx, Wq, dw, Y, workspace=None):
     wsb = workspace.numel() * workspace.element_size() if workspace is not None else 0
     _check(load().smoothrot_linear(xp, _vec(dx, M, "dx"), M, wp, _vec(dw, N, "dw"), N, K, yp, ldy,
                                    wsp, wsb, _stream()))
+
+
+STATIC_SCRATCH_BYTES = 8 * 1024 * 1024   # SMOOTHROT_STATIC_SCRATCH_BYTES in the header
+
+
+def linear_static_scratch(Xq, dx, Wq, dw, Y):
+    """smoothrot_linear_static_scratch: same result as linear(), for callers that cannot
+    hand over a workspace.  The split-K scratch is a fixed array inside the library (one per
+    device, shared by all calls: do not let two calls overlap on the GPU).  Shapes that need
+    more than STATIC_SCRATCH_BYTES raise SmoothRotError (status -7).  Allocates nothing."""
+    xp, M, K = _packed(Xq, "Xq")
+    wp, N, Kw = _packed(Wq, "Wq")
+    if K != Kw:
+        raise ValueError("Xq and Wq disagree on K")
+    yp, My, Ny, ldy = _rows(Y, torch.float16, "Y")
+    if (My, Ny) != (M, N):
+        raise ValueError(f"Y must be [{M}, {N}]")
+    _check(load().smoothrot_linear_static_scratch(xp, _vec(dx, M, "dx"), M, wp, _vec(dw, N, "dw"), N, K,
+                                                  yp, ldy, _stream()))
 
 
 def debug_hadamard(X, pre, Y):

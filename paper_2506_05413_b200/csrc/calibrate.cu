@@ -110,6 +110,8 @@ const char* smoothrot_status_string(int status) {
     case SMOOTHROT_WORKSPACE_TOO_SMALL: return "workspace too small";
     case SMOOTHROT_CUDA_ERROR: return "CUDA error";
     case SMOOTHROT_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+    case SMOOTHROT_STATIC_SCRATCH_EXCEEDED:
+      return "shape needs more split-K scratch than the library's built-in array holds";
     default: return "unknown status";
   }
 }

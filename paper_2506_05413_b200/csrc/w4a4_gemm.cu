@@ -626,10 +626,61 @@ static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq,
   return rc;
 }
 
+// ---------------------------------------------------------------------------
+// Built-in scratch for smoothrot_linear_static_scratch: split-K partial sums
+// for callers that have no way to provide a workspace of their own.  The array
+// is part of the loaded module, so every device that loads the library holds
+// these bytes until the process exits.
+// ---------------------------------------------------------------------------
+constexpr size_t kStaticScratchBytes = size_t(SMOOTHROT_STATIC_SCRATCH_BYTES);
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static std::atomic<void*> g_static_scratch_addr[kMaxDevices];
+
+// Device address of g_static_scratch on the current device.  In host code the
+// array's name is only a handle for the runtime; the address a kernel can use
+// has to be asked for, once per device, with that device current.
+static int static_scratch_address(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SMOOTHROT_CUDA_ERROR;
+  void* p = g_static_scratch_addr[dev].load(std::memory_order_acquire);
+  if (p == nullptr) {
+    void* sym = nullptr;
+    if (cudaGetSymbolAddress(&sym, g_static_scratch) != cudaSuccess || sym == nullptr) {
+      (void)cudaGetLastError();
+      return SMOOTHROT_CUDA_ERROR;
+    }
+    g_static_scratch_addr[dev].store(sym, std::memory_order_release);
+    p = sym;
+  }
+  *out = p;
+  return SMOOTHROT_OK;
+}
+
 }  // namespace gemm
 }  // namespace smoothrot
 
 extern "C" {
+
+int smoothrot_linear_static_scratch(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq,
+                                    const float* dw, int64_t N, int64_t K, void* Y_f16, int64_t ldy,
+                                    void* stream) {
+  using namespace smoothrot::gemm;
+  if (M > 0 && N > 0 && Y_f16 == nullptr) return SMOOTHROT_INVALID_ARG;
+  const size_t need = smoothrot_workspace_bytes(M, N, K);
+  if (need > kStaticScratchBytes) return SMOOTHROT_STATIC_SCRATCH_EXCEEDED;
+  void* scratch = nullptr;
+  if (need > 0) {
+    const int rc = static_scratch_address(&scratch);
+    if (rc != SMOOTHROT_OK) return rc;
+  }
+  // Every partial sum the reduction reads is written by the GEMM kernel of the
+  // same call, so nothing left in the array by an earlier call is ever read
+  // and nothing has to be cleared.
+  return run(Xq, dx, M, Wq, dw, N, K, static_cast<__half*>(Y_f16), ldy, nullptr, scratch,
+             need > 0 ? kStaticScratchBytes : 0, static_cast<cudaStream_t>(stream));
+}
 
 size_t smoothrot_workspace_bytes(int64_t M, int64_t N, int64_t K) {
   if (M <= 0 || N <= 0 || K <= 0 || K % smoothrot::gemm::kWideRow != 0) return 0;
