@@ -12,31 +12,54 @@ namespace smoothrot {
 
 std::atomic<int64_t> g_launches{0};
 
-constexpr int kAbsmaxThreads = 128;   // each thread owns 8 adjacent channels
+constexpr int kAbsmaxChunks = 128;     // 8-channel chunks per CTA (x dimension of the block)
+constexpr int kAbsmaxRowLanes = 4;     // threads that share a chunk and split the rows (y dimension)
 constexpr int kAbsmaxRowsPerCta = 64;
 
-__global__ void __launch_bounds__(kAbsmaxThreads)
-column_absmax_kernel(const __half* __restrict__ X, int64_t rows, int64_t K, int64_t ld,
-                     float* __restrict__ amax) {
-  const int64_t c8 = int64_t(blockIdx.x) * kAbsmaxThreads + threadIdx.x;  // 8-channel chunk
-  if (c8 * 8 >= K) return;
-  const int64_t r0 = int64_t(blockIdx.y) * kAbsmaxRowsPerCta;
-  const int64_t r1 = min(rows, r0 + kAbsmaxRowsPerCta);
+__device__ __forceinline__ void absmax_fold(uint4& best, const uint4& v) {
   // |x| as fp16 bit patterns: clear the sign bits, then a packed unsigned max
   // on the 16-bit lanes orders the magnitudes (NaNs aside).
+  best.x = __vmaxu2(best.x, v.x & 0x7fff7fffu);
+  best.y = __vmaxu2(best.y, v.y & 0x7fff7fffu);
+  best.z = __vmaxu2(best.z, v.z & 0x7fff7fffu);
+  best.w = __vmaxu2(best.w, v.w & 0x7fff7fffu);
+}
+
+__global__ void __launch_bounds__(kAbsmaxChunks * kAbsmaxRowLanes)
+column_absmax_kernel(const __half* __restrict__ X, int64_t rows, int64_t K, int64_t ld,
+                     float* __restrict__ amax) {
+  __shared__ uint4 part[kAbsmaxRowLanes][kAbsmaxChunks];
+  const int64_t c8 = int64_t(blockIdx.x) * kAbsmaxChunks + threadIdx.x;  // 8-channel chunk
+  const bool live = c8 * 8 < K;
+  const int64_t r0 = int64_t(blockIdx.y) * kAbsmaxRowsPerCta + threadIdx.y;
+  const int64_t r1 = min(rows, int64_t(blockIdx.y + 1) * kAbsmaxRowsPerCta);
   uint4 best = make_uint4(0u, 0u, 0u, 0u);
-  for (int64_t r = r0; r < r1; ++r) {
-    uint4 v = __ldg(reinterpret_cast<const uint4*>(X + r * ld + c8 * 8));
-    best.x = __vmaxu2(best.x, v.x & 0x7fff7fffu);
-    best.y = __vmaxu2(best.y, v.y & 0x7fff7fffu);
-    best.z = __vmaxu2(best.z, v.z & 0x7fff7fffu);
-    best.w = __vmaxu2(best.w, v.w & 0x7fff7fffu);
+  if (live) {
+    const __half* col = X + c8 * 8;
+    int64_t r = r0;
+    // eight independent 16-byte loads in flight per thread
+    for (; r + 7 * kAbsmaxRowLanes < r1; r += 8 * kAbsmaxRowLanes) {
+      uint4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        v[u] = __ldg(reinterpret_cast<const uint4*>(col + (r + u * kAbsmaxRowLanes) * ld));
+#pragma unroll
+      for (int u = 0; u < 8; ++u) absmax_fold(best, v[u]);
+    }
+    for (; r < r1; r += kAbsmaxRowLanes)
+      absmax_fold(best, __ldg(reinterpret_cast<const uint4*>(col + r * ld)));
   }
+  part[threadIdx.y][threadIdx.x] = best;
+  __syncthreads();
+  if (threadIdx.y != 0 || !live) return;
+#pragma unroll
+  for (int y = 1; y < kAbsmaxRowLanes; ++y) absmax_fold(best, part[y][threadIdx.x]);
   const __half2* h = reinterpret_cast<const __half2*>(&best);
   int* out = reinterpret_cast<int*>(amax + c8 * 8);
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const float2 f = __half22float2(h[i]);
+    // non-negative floats order like their bit patterns
     atomicMax(out + 2 * i, __float_as_int(f.x));
     atomicMax(out + 2 * i + 1, __float_as_int(f.y));
   }
@@ -61,9 +84,10 @@ __global__ void finalize_scales_kernel(const float* __restrict__ amax, float* __
 }
 
 static void launch_absmax(const __half* X, int64_t rows, int64_t K, int64_t ld, float* amax, cudaStream_t st) {
-  dim3 grid(unsigned((K / 8 + kAbsmaxThreads - 1) / kAbsmaxThreads),
+  dim3 grid(unsigned((K / 8 + kAbsmaxChunks - 1) / kAbsmaxChunks),
             unsigned((rows + kAbsmaxRowsPerCta - 1) / kAbsmaxRowsPerCta));
-  column_absmax_kernel<<<grid, kAbsmaxThreads, 0, st>>>(X, rows, K, ld, amax);
+  dim3 block(kAbsmaxChunks, kAbsmaxRowLanes);
+  column_absmax_kernel<<<grid, block, 0, st>>>(X, rows, K, ld, amax);
   count_launch();
 }
 

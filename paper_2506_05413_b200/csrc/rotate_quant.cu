@@ -232,23 +232,64 @@ __device__ __forceinline__ void group_barrier(int group) {
   asm volatile("bar.sync %0, 64;" ::"r"(group + 1) : "memory");
 }
 
-template <int N>
-__device__ __forceinline__ void butterflies_inplace(float* v) {
+// Two fp32 values in one 64-bit register, for the packed add/sub/mul/fma of sm_100.
+typedef unsigned long long f32x2;
+
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+  f32x2 r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) {
+  f32x2 r;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+  f32x2 r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+
+// Walsh butterflies on 2 * NP values held as NP pairs (pair k = values 2k, 2k+1).
+// The stage inside a pair is scalar; every other stage works on whole pairs.
+template <int NP>
+__device__ __forceinline__ void butterflies_pairs(f32x2* v) {
 #pragma unroll
-  for (int h = 1; h < N; h <<= 1) {
+  for (int k = 0; k < NP; ++k) {
+    float a, b;
+    unpack2(v[k], a, b);
+    v[k] = pack2(a + b, a - b);
+  }
 #pragma unroll
-    for (int i = 0; i < N; ++i) {
-      if ((i & h) == 0) {
-        float a = v[i], b = v[i + h];
-        v[i] = a + b;
-        v[i + h] = a - b;
+  for (int h = 1; h < NP; h <<= 1) {
+#pragma unroll
+    for (int k = 0; k < NP; ++k) {
+      if ((k & h) == 0) {
+        const f32x2 a = v[k], b = v[k + h];
+        v[k] = add2(a, b);
+        v[k + h] = sub2(a, b);
       }
     }
   }
 }
 
-template <bool kQuant, bool kHasPre>
-__global__ void __launch_bounds__(kW4096Rows * 64)
+// kLowClamp: whether codes below -8 can occur (only for clip ratios <= 7/8.5).
+template <bool kQuant, bool kHasPre, bool kLowClamp>
+__global__ void __launch_bounds__(kW4096Rows * 64, 3)
 walsh4096_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
                  const float* __restrict__ pre, float clip,
                  uint8_t* __restrict__ q_out, float* __restrict__ step_out,
@@ -262,7 +303,9 @@ walsh4096_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
   if (m >= M) return;  // whole row group leaves together; only group barriers are used
   float* tile = smem + group * (64 * kW4096Pitch);
 
-  float v[64];
+  // The values stay unnormalised until the end: 1/sqrt(4096) = 2^-6 is exact,
+  // so it is folded into the step size (or applied at the fp32 store).
+  f32x2 v[32];
   {
     const __half* x = X + m * ldx;
     uint4 raw[8];
@@ -270,65 +313,93 @@ walsh4096_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
     for (int g = 0; g < 8; ++g) raw[g] = __ldg(reinterpret_cast<const uint4*>(x + g * 512 + t * 8));
 #pragma unroll
     for (int g = 0; g < 8; ++g) {
-      unpack8_f16(raw[g], &v[g * 8]);
+      const __half2* h = reinterpret_cast<const __half2*>(&raw[g]);
+      float4 p0, p1;
       if (kHasPre) {
-        const float4 p0 = __ldg(reinterpret_cast<const float4*>(pre + g * 512 + t * 8));
-        const float4 p1 = __ldg(reinterpret_cast<const float4*>(pre + g * 512 + t * 8 + 4));
-        v[g * 8 + 0] *= p0.x * 0.015625f; v[g * 8 + 1] *= p0.y * 0.015625f;
-        v[g * 8 + 2] *= p0.z * 0.015625f; v[g * 8 + 3] *= p0.w * 0.015625f;
-        v[g * 8 + 4] *= p1.x * 0.015625f; v[g * 8 + 5] *= p1.y * 0.015625f;
-        v[g * 8 + 6] *= p1.z * 0.015625f; v[g * 8 + 7] *= p1.w * 0.015625f;
-      } else {
+        p0 = __ldg(reinterpret_cast<const float4*>(pre + g * 512 + t * 8));
+        p1 = __ldg(reinterpret_cast<const float4*>(pre + g * 512 + t * 8 + 4));
+      }
 #pragma unroll
-        for (int i = 0; i < 8; ++i) v[g * 8 + i] *= 0.015625f;
+      for (int k = 0; k < 4; ++k) {
+        const float2 f = __half22float2(h[k]);
+        f32x2 val = pack2(f.x, f.y);
+        if (kHasPre) {
+          const f32x2 pp = k == 0 ? pack2(p0.x, p0.y) : k == 1 ? pack2(p0.z, p0.w)
+                         : k == 2 ? pack2(p1.x, p1.y) : pack2(p1.z, p1.w);
+          val = mul2(val, pp);
+        }
+        v[g * 4 + k] = val;
       }
     }
   }
-  butterflies_inplace<64>(v);  // v index = g * 8 + i: bits of i, then bits of g
+  butterflies_pairs<32>(v);  // value index = g * 8 + i: bits of i, then bits of g
 
   // transpose: thread t writes its 64 values as one padded row
   {
     float4* dst = reinterpret_cast<float4*>(tile + t * kW4096Pitch);
 #pragma unroll
-    for (int c = 0; c < 16; ++c) dst[c] = make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+    for (int c = 0; c < 16; ++c) {
+      float4 o;
+      unpack2(v[2 * c], o.x, o.y);
+      unpack2(v[2 * c + 1], o.z, o.w);
+      dst[c] = o;
+    }
   }
   group_barrier(group);
   // thread gi = t now owns position (g, i) = (t >> 3, t & 7) for all 64 values of the t-bits
 #pragma unroll
-  for (int u = 0; u < 64; ++u) v[u] = tile[u * kW4096Pitch + t];
-  butterflies_inplace<64>(v);
+  for (int u = 0; u < 32; ++u) v[u] = pack2(tile[(2 * u) * kW4096Pitch + t], tile[(2 * u + 1) * kW4096Pitch + t]);
+  butterflies_pairs<32>(v);
 
   const int gi_g = t >> 3, gi_i = t & 7;
   if (!kQuant) {
     float* y = y_out + m * 4096;
 #pragma unroll
-    for (int u = 0; u < 64; ++u) y[gi_g * 512 + u * 8 + gi_i] = v[u];
+    for (int u = 0; u < 32; ++u) {
+      float a, b;
+      unpack2(v[u], a, b);
+      y[gi_g * 512 + (2 * u) * 8 + gi_i] = a * 0.015625f;
+      y[gi_g * 512 + (2 * u + 1) * 8 + gi_i] = b * 0.015625f;
+    }
     return;
   }
 
   float amax = 0.0f;
 #pragma unroll
-  for (int u = 0; u < 64; ++u) amax = fmaxf(amax, fabsf(v[u]));
+  for (int u = 0; u < 32; ++u) {
+    float a, b;
+    unpack2(v[u], a, b);
+    amax = fmaxf(amax, fmaxf(fabsf(a), fabsf(b)));
+  }
   amax = warp_max(amax);
   if (lane == 0) red[group][t >> 5] = amax;
   group_barrier(group);
-  amax = fmaxf(red[group][0], red[group][1]);
+  amax = fmaxf(red[group][0], red[group][1]) * 0.015625f;   // now the absmax of the normalised row
   const float step = step_from_absmax(amax, clip);
   if (t == 0) step_out[m] = step;
-  const float inv = __frcp_rn(step);
+  const float inv = __frcp_rn(step) * 0.015625f;            // 1/step for unnormalised values (exact scaling)
+  const f32x2 inv2 = pack2(inv, inv);
 
   // Round to nearest even and bias by 8: the low byte of the float's bit
   // pattern is code + 8 in [0, 15].
   const float kMagic = 12582912.0f + 8.0f;  // 1.5 * 2^23 + 8
+  const f32x2 magic2 = pack2(kMagic, kMagic);
   uint32_t spread[16];                      // four codes per word, one per byte
 #pragma unroll
   for (int c = 0; c < 16; ++c) {
     uint32_t r[4];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      float q = fmaf(v[4 * c + k], inv, kMagic);
-      q = fminf(fmaxf(q, 12582912.0f), 12582912.0f + 15.0f);
-      r[k] = __float_as_uint(q);
+    for (int k = 0; k < 2; ++k) {
+      float q0, q1;
+      unpack2(fma2(v[2 * c + k], inv2, magic2), q0, q1);
+      q0 = fminf(q0, 12582912.0f + 15.0f);
+      q1 = fminf(q1, 12582912.0f + 15.0f);
+      if (kLowClamp) {
+        q0 = fmaxf(q0, 12582912.0f);
+        q1 = fmaxf(q1, 12582912.0f);
+      }
+      r[2 * k] = __float_as_uint(q0);
+      r[2 * k + 1] = __float_as_uint(q1);
     }
     const uint32_t lo = __byte_perm(r[0], r[1], 0x0040);  // bytes: r0.b0, r1.b0
     const uint32_t hi = __byte_perm(r[2], r[3], 0x0040);
@@ -390,8 +461,12 @@ static int launch_rotate(const void* X, int64_t rows, int64_t K, int64_t ld, con
   const __half* x = static_cast<const __half*>(X);
   if (K == 4096) {
     const size_t smem = size_t(kW4096Rows) * 64 * kW4096Pitch * sizeof(float);
-    auto kern = pre ? walsh4096_kernel<kQuant, true> : walsh4096_kernel<kQuant, false>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
+    // codes below -8 can only come up when the row maximum sits at 8.5 steps or more
+    const bool low = kQuant && (7.0f / clip >= 8.49f);
+    auto kern = pre ? (low ? walsh4096_kernel<kQuant, true, true> : walsh4096_kernel<kQuant, true, false>)
+                    : (low ? walsh4096_kernel<kQuant, false, true> : walsh4096_kernel<kQuant, false, false>);
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess ||
+        cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, 100) != cudaSuccess)
       return SMOOTHROT_CUDA_ERROR;
     const unsigned grid = unsigned((rows + kW4096Rows - 1) / kW4096Rows);
     kern<<<grid, kW4096Rows * 64, smem, stream>>>(x, ld, rows, pre, clip, q_out, step_out, y_out);

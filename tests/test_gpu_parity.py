@@ -100,6 +100,21 @@ def test_quantized_codes_match_oracle(gu, K, M, which):
     assert codes.min() >= -8 and codes.max() <= 7
 
 
+@pytest.mark.parametrize("K", [512, 4096, 14336])
+@pytest.mark.parametrize("clip", [0.5, 0.8, 0.83, 1.0])
+def test_quantizer_clip_ratios_including_two_sided_saturation(gu, K, clip):
+    """Below clip = 7/8.5 values can fall under -8.5 steps and must saturate at -8."""
+    from paper_2506_05413_b200 import binding as sr
+    X = _acts(K + int(100 * clip), 23, K, gain=30.0)
+    q, step = gu.gpu_quantize(sr.quant_act, X, None, clip)
+    q_ref, step_ref, _ = orc.quant_act(X, None, K, clip)
+    assert np.abs(step / step_ref - 1).max() <= TOL_SCALE
+    frac, worst = gu.code_mismatch(q, q_ref)
+    assert worst <= 1 and frac <= TOL_CODES
+    if clip <= 0.8:
+        assert orc.unpack_codes(q_ref).min() == -8 and orc.unpack_codes(q_ref).max() == 7
+
+
 def test_quantizer_edge_rows(gu):
     from paper_2506_05413_b200 import binding as sr
     for K in (128, 4096, 14336):
