@@ -162,6 +162,8 @@ GEMM_SHAPES = [
     (130, 136, 640),     # BN = 128, ragged both ways
     (300, 520, 1152),    # BN = 256, several tiles and a ragged tail
     (257, 8, 128),
+    (256, 256, 128),     # one two-CTA pair tile
+    (600, 776, 512),     # two-CTA tiles, ragged in both directions
     (512, 1024, 14336),  # long K
 ]
 
@@ -186,7 +188,8 @@ def test_gemm_extreme_codes(gu):
     assert np.all(got[:, 0::2] == 64 * K) and np.all(got[:, 1::2] == -56 * K)
 
 
-@pytest.mark.parametrize("M,N,K", [(64, 256, 128), (3, 1024, 4096), (200, 264, 512), (130, 520, 4096)])
+@pytest.mark.parametrize("M,N,K", [(64, 256, 128), (3, 1024, 4096), (200, 264, 512), (130, 520, 4096),
+                                   (300, 520, 640), (1024, 768, 4096)])
 def test_linear_output_matches_oracle_on_gpu_codes(gu, M, N, K):
     rng = np.random.default_rng(M + N + K)
     xq = orc.pack_codes(synth.random_codes(M, M, K))
