@@ -496,8 +496,14 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
   return r;
 }
+// Arrival on a barrier of the other CTA of the pair.  The data this signals
+// (int8 tiles in the arriving CTA's own shared memory, already fenced for the
+// async proxy; accumulator reads already fenced with tcgen05.fence) is consumed
+// by tensor-core work on the arriving CTA's own SM, so the default CTA-scope
+// release is enough; a cluster-scope release here stalls every arriving warp
+// for well over a thousand cycles per k-block.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
