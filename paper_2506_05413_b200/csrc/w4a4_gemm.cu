@@ -723,6 +723,374 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
   }
 }
 
+// ---------------------------------------------------------------------------
+// Two-CTA kernel with the token operand in tensor memory.
+//
+// Shared-memory bandwidth (128 bytes per clock and SM, shared by TMA writes,
+// the widen warps and the tensor core's operand reads) is what bounds the
+// kernels above.  Here the A side (128 token rows per CTA) never goes back to
+// shared memory after it was widened: "A-widen" warps read the packed rows
+// that TMA delivered, widen them in registers and write them with tcgen05.st
+// into a ring of slots in tensor memory, from where tcgen05.mma takes its A
+// operand.  Only the B side (each CTA's half of the 256 output channels) is
+// widened into shared memory.  Per 128-deep k-block a CTA then moves
+// 16 KB (A: TMA write + read) + 48 KB (B: TMA write, read, int8 write,
+// tensor-core read) through shared memory, against 96 KB before.
+//
+// Tensor memory: columns [0, 256) hold the one 128 x 256 int32 accumulator,
+// columns [256, 256 + 32 * kStages) the A ring (a k-block of a row is 128 int8
+// = 32 columns).  With a single accumulator the epilogue cannot overlap the
+// next tile's MMAs; it drains the accumulator into a shared-memory staging
+// area as fp16 (releasing tensor memory as soon as the last tcgen05.ld has
+// returned) and TMA stores write the staged tile to Y asynchronously.
+// ---------------------------------------------------------------------------
+struct PairT {
+  static constexpr int kBN = 256;      // output channels per pair tile
+  static constexpr int kHalfN = 128;   // B-side rows staged by each CTA
+  static constexpr int kStages = 5;    // int8 B stages in shared memory = A slots in tensor memory
+  static constexpr int kPackedStages = 4;
+  static constexpr int kPackedA = kBM * kPackedRow, kPackedB = kHalfN * kPackedRow;
+  static constexpr int kPackedStageBytes = kPackedA + kPackedB;
+  static constexpr int kWideB = kHalfN * kWideRow;
+  static constexpr int kOutBoxBytes = 32 * 128;              // 32 rows x 64 fp16
+  static constexpr int kOutBytes = kEpiWarps * 4 * kOutBoxBytes;  // 128 rows x 256 fp16
+  static constexpr int kNumBarriers = 2 * kStages + 2 * kPackedStages + 2;
+  static constexpr int kSmemBytes = 1024 + kStages * kWideB + kPackedStages * kPackedStageBytes + kOutBytes +
+                                    kNumBarriers * 8 + 16;
+  static constexpr int kTmemCols = 512;
+  static constexpr int kAccCols = 256;
+  static constexpr int kAWidenWarps = 4, kBWidenWarps = 4;
+  static_assert(kAccCols + 32 * kStages <= kTmemCols, "A ring does not fit tensor memory");
+  static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
+  static_assert(kAWidenWarps + kBWidenWarps == kWidenWarps, "warp roles");
+};
+
+__device__ __forceinline__ void mma_i8_pair_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// 32 consecutive 32-bit columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_store32(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Waits until the shared-memory sources of all earlier bulk stores of this thread have been read.
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                           const __grid_constant__ CUtensorMap map_y, const Params p) {
+  using T = PairT;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t base = (raw_addr + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - raw_addr);
+
+  const uint32_t wide_base = base;                                             // int8 B stages
+  const uint32_t packed_base = wide_base + T::kStages * T::kWideB;             // packed A + B stages
+  const uint32_t out_base = packed_base + T::kPackedStages * T::kPackedStageBytes;  // fp16 output staging
+  const uint32_t bar_base = out_base + T::kOutBytes;
+  // full[s]: A slot s written in both CTAs' tensor memory and B stage s written in both CTAs' shared
+  // memory (collected in the leader); empty[s]: the MMAs that read them have completed (both CTAs).
+  auto full = [&](int s) { return bar_base + 8u * s; };
+  auto empty = [&](int s) { return bar_base + 8u * (T::kStages + s); };
+  auto pk_full = [&](int s) { return bar_base + 8u * (2 * T::kStages + s); };
+  auto pk_empty = [&](int s) { return bar_base + 8u * (2 * T::kStages + T::kPackedStages + s); };
+  const uint32_t acc_full = bar_base + 8u * (2 * T::kStages + 2 * T::kPackedStages);
+  const uint32_t acc_empty = acc_full + 8u;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + (bar_base - base) + 8 * T::kNumBarriers);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < T::kStages; ++s) {
+      mbar_init(full(s), 2 * kWidenWarps);   // A-widen and B-widen warps of both CTAs (used in the leader only)
+      mbar_init(empty(s), 1);
+    }
+    for (int s = 0; s < T::kPackedStages; ++s) {
+      mbar_init(pk_full(s), 1);
+      mbar_init(pk_empty(s), kWidenWarps);
+    }
+    mbar_init(acc_full, 1);
+    mbar_init(acc_empty, 2 * kEpiWarps);     // epilogue warps of both CTAs (used in the leader only)
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async();
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(tmem_slot)), "r"(uint32_t(T::kTmemCols)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  tcgen05_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_a_ring = tmem_base + uint32_t(T::kAccCols);
+
+  const int total_tiles = p.tiles_a * p.tiles_b;
+  const int first_tile = blockIdx.x >> 1;
+  const int tile_step = gridDim.x >> 1;
+  const int kblocks = p.kblocks;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (each CTA, own rows)
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
+        const int ta = tile % p.tiles_a;
+        const int tb = tile / p.tiles_a;
+        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+          const int s = it % T::kPackedStages;
+          const uint32_t ph = (it / T::kPackedStages) & 1u;
+          if (!mbar_wait(pk_empty(s), ph ^ 1u, abort_flag, kSiteProducer)) { ok = false; break; }
+          mbar_expect_tx(pk_full(s), uint32_t(T::kPackedA + T::kPackedB));
+          const uint32_t dst = packed_base + s * T::kPackedStageBytes;
+          tma_load_2d(dst, &map_a, pk_full(s), kb * kPackedRow, ta * 256 + int(rank) * kBM);
+          tma_load_2d(dst + T::kPackedA, &map_b, pk_full(s), kb * kPackedRow, tb * T::kBN + int(rank) * T::kHalfN);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (leader && lane == 0) {
+      constexpr uint32_t idesc = make_idesc_i8_pair(T::kBN);
+      uint32_t it = 0, local_tile = 0;
+      bool ok = true;
+      for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step, ++local_tile) {
+        if (!mbar_wait(acc_empty, (local_tile & 1u) ^ 1u, abort_flag, kSiteMmaAcc)) break;
+        tcgen05_fence_after();
+        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+          const int s = it % T::kStages;
+          const uint32_t ph = (it / T::kStages) & 1u;
+          if (!mbar_wait(full(s), ph, abort_flag, kSiteMmaWide)) { ok = false; break; }
+          tcgen05_fence_after();
+          const uint64_t db = make_desc_sw128(wide_base + s * T::kWideB);
+          const uint32_t ta_addr = tmem_a_ring + uint32_t(s * 32);
+#pragma unroll
+          for (int k4 = 0; k4 < 4; ++k4)   // 32 int8 of K: 8 columns of A, 32 bytes of B's swizzle atom
+            mma_i8_pair_ts(tmem_base, ta_addr + uint32_t(8 * k4), db + uint64_t(2 * k4), idesc,
+                           (kb > 0 || k4 > 0) ? 1u : 0u);
+          tcgen05_commit_pair(empty(s));
+        }
+        if (ok) tcgen05_commit_pair(acc_full);
+      }
+    }
+  } else if (warp < 2 + T::kAWidenWarps) {
+    // ------------------------------------------------------------ A-widen warps: packed rows -> tensor memory
+    const int q = warp & 3;               // tensor-memory lane quadrant this warp may write
+    const int row = q * 32 + lane;        // A row inside the CTA's 128 = tensor-memory lane
+    const uint32_t sw = uint32_t((row >> 1) & 3);
+    uint32_t it = 0;
+    bool ok = true;
+    for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
+      for (int kb = 0; kb < kblocks; ++kb, ++it) {
+        const int ps = it % T::kPackedStages;
+        const uint32_t pph = (it / T::kPackedStages) & 1u;
+        const int s = it % T::kStages;
+        const uint32_t sph = (it / T::kStages) & 1u;
+        if (!mbar_wait(pk_full(ps), pph, abort_flag, kSiteWidenFull)) { ok = false; break; }
+        const uint32_t src = packed_base + ps * T::kPackedStageBytes + row * kPackedRow;
+        uint32_t x[16];
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                       : "=r"(x[4 * c]), "=r"(x[4 * c + 1]), "=r"(x[4 * c + 2]), "=r"(x[4 * c + 3])
+                       : "r"(src + ((uint32_t(c) ^ sw) << 4)) : "memory");
+        // Same order of k inside a k-block as the B side: per 32 packed codes, the 16 even codes
+        // (low nibbles) first, then the 16 odd codes.
+        uint32_t r[32];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            r[8 * c + i] = (x[4 * c + i] << 4) & 0xF0F0F0F0u;
+            r[8 * c + 4 + i] = x[4 * c + i] & 0xF0F0F0F0u;
+          }
+        }
+        if (!mbar_wait(empty(s), sph ^ 1u, abort_flag, kSiteWidenEmpty)) { ok = false; break; }
+        tcgen05_fence_after();
+        tmem_store32(tmem_a_ring + (uint32_t(q * 32) << 16) + uint32_t(s * 32), r);
+        tmem_wait_st();
+        tcgen05_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          if (leader) mbar_arrive(full(s));
+          else mbar_arrive_cluster(map_to_cta(full(s), 0));
+          mbar_arrive(pk_empty(ps));
+        }
+      }
+    }
+  } else if (warp < 2 + kWidenWarps) {
+    // ------------------------------------------------------------ B-widen warps: packed rows -> int8 tile
+    const int w = warp - 2 - T::kAWidenWarps;
+    const int r = lane & 7;
+    const int c = lane >> 3;
+    constexpr int kGroups = T::kHalfN / 8;
+    uint32_t it = 0;
+    bool ok = true;
+    for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
+      for (int kb = 0; kb < kblocks; ++kb, ++it) {
+        const int ps = it % T::kPackedStages;
+        const uint32_t pph = (it / T::kPackedStages) & 1u;
+        const int s = it % T::kStages;
+        const uint32_t sph = (it / T::kStages) & 1u;
+        if (!mbar_wait(pk_full(ps), pph, abort_flag, kSiteWidenFull)) { ok = false; break; }
+        if (!mbar_wait(empty(s), sph ^ 1u, abort_flag, kSiteWidenEmpty)) { ok = false; break; }
+        const uint32_t pk = packed_base + ps * T::kPackedStageBytes + T::kPackedA;
+        const uint32_t wd = wide_base + s * T::kWideB;
+#pragma unroll
+        for (int g = w; g < kGroups; g += T::kBWidenWarps) {
+          const int row = g * 8 + r;
+          const uint32_t src = pk + row * kPackedRow + ((c ^ ((row >> 1) & 3)) << 4);
+          const uint32_t dst_row = wd + row * kWideRow;
+          uint32_t x0, x1, x2, x3;
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                       : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3) : "r"(src) : "memory");
+          const uint32_t lo_dst = dst_row + (((2 * c) ^ (row & 7)) << 4);
+          const uint32_t hi_dst = dst_row + (((2 * c + 1) ^ (row & 7)) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                       ::"r"(lo_dst), "r"((x0 << 4) & 0xF0F0F0F0u), "r"((x1 << 4) & 0xF0F0F0F0u),
+                         "r"((x2 << 4) & 0xF0F0F0F0u), "r"((x3 << 4) & 0xF0F0F0F0u) : "memory");
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                       ::"r"(hi_dst), "r"(x0 & 0xF0F0F0F0u), "r"(x1 & 0xF0F0F0F0u),
+                         "r"(x2 & 0xF0F0F0F0u), "r"(x3 & 0xF0F0F0F0u) : "memory");
+        }
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) {
+          if (leader) mbar_arrive(full(s));
+          else mbar_arrive_cluster(map_to_cta(full(s), 0));
+          mbar_arrive(pk_empty(ps));
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue warps (each CTA, own 128 rows)
+    const int q = warp & 3;               // tensor-memory lane quadrant this warp may read
+    const uint32_t out_warp = out_base + uint32_t(q) * uint32_t(4 * T::kOutBoxBytes);
+    const uint32_t taddr = tmem_base + (uint32_t(q * 32) << 16);
+    uint32_t local_tile = 0;
+    for (int tile = first_tile; tile < total_tiles; tile += tile_step, ++local_tile) {
+      const int ta = tile % p.tiles_a;
+      const int tb = tile / p.tiles_a;
+      if (!mbar_wait(acc_full, local_tile & 1u, abort_flag, kSiteEpilogue)) break;
+      tcgen05_fence_after();
+      const int row0 = ta * 256 + int(rank) * kBM + q * 32;
+      const int a = row0 + lane;
+      if (p.Y != nullptr) {
+        // the staging boxes of the previous tile must have been read by their TMA stores
+        if (lane == 0) tma_store_wait_read();
+        __syncwarp();
+        const float sx = a < p.rows_a ? __ldg(p.dx + a) * 0.00390625f : 0.0f;   // accumulators are 256 * acc
+#pragma unroll 1
+        for (int cb = 0; cb < 4; ++cb) {
+          const uint32_t box = out_warp + uint32_t(cb * T::kOutBoxBytes);
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            uint32_t regs[32];
+            tmem_load32(taddr + uint32_t(cb * 64 + h * 32), regs);
+            tmem_wait_ld();
+            if (cb == 3 && h == 1) {
+              // the accumulator is in registers or staged: hand tensor memory back to the MMA warp
+              tcgen05_fence_before();
+              __syncwarp();
+              if (lane == 0) {
+                if (leader) mbar_arrive(acc_empty);
+                else mbar_arrive_cluster(map_to_cta(acc_empty, 0));
+              }
+            }
+            const int n0 = tb * T::kBN + cb * 64 + h * 32;
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+              const int n = n0 + 8 * jj;
+              float4 w0 = make_float4(0.f, 0.f, 0.f, 0.f), w1 = w0;
+              if (n + 8 <= p.rows_b) {
+                w0 = __ldg(reinterpret_cast<const float4*>(p.dw + n));
+                w1 = __ldg(reinterpret_cast<const float4*>(p.dw + n + 4));
+              }
+              const float ws[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+              uint32_t o[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float v0 = float(int32_t(regs[8 * jj + 2 * e])) * (sx * ws[2 * e]);
+                const float v1 = float(int32_t(regs[8 * jj + 2 * e + 1])) * (sx * ws[2 * e + 1]);
+                const __half2 hv = __floats2half2_rn(v0, v1);
+                o[e] = *reinterpret_cast<const uint32_t*>(&hv);
+              }
+              const uint32_t chunk = uint32_t(h * 4 + jj) ^ uint32_t(lane & 7);   // 128-byte swizzle of the store map
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                           ::"r"(box + uint32_t(lane) * 128u + (chunk << 4)), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3])
+                           : "memory");
+            }
+          }
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {
+            const int x = tb * T::kBN + cb * 64;
+            if (x < p.rows_b && row0 < p.rows_a) tma_store_2d(&map_y, box, x, row0);   // TMA clips the ragged edges
+          }
+        }
+        if (lane == 0) tma_store_commit();
+      } else {
+        // test export of the int32 accumulators: plain stores
+#pragma unroll 1
+        for (int c0 = 0; c0 < T::kBN; c0 += 32) {
+          uint32_t regs[32];
+          tmem_load32(taddr + uint32_t(c0), regs);
+          tmem_wait_ld();
+          store_columns<32>(p, a, tb * T::kBN + c0, 0, regs);
+          __syncwarp();
+        }
+        tcgen05_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          if (leader) mbar_arrive(acc_empty);
+          else mbar_arrive_cluster(map_to_cta(acc_empty, 0));
+        }
+      }
+    }
+    if (lane == 0) tma_store_wait_all();
+  }
+
+  tcgen05_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // both CTAs are done with both halves of tensor memory
+  if (warp == 1) {
+    __syncwarp();
+    tcgen05_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;"
+                 ::"r"(tmem_base), "r"(uint32_t(T::kTmemCols)) : "memory");
+  }
+}
+
 // Sums the split-K partials and applies the dequantization (or writes the int32 sum).
 __global__ void splitk_reduce_kernel(const int32_t* __restrict__ part, int splits, int M, int N,
                                      const float* __restrict__ dx, const float* __restrict__ dw,
@@ -815,6 +1183,19 @@ static bool make_map(CUtensorMap* map, const uint8_t* ptr, int64_t rows, int64_t
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 2-D map over the fp16 output [M x ldy], box = 64 columns x 32 rows, 128-byte swizzle (TMA stores).
+static bool make_map_y(CUtensorMap* map, __half* Y, int64_t M, int64_t N, int64_t ldy) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  const cuuint64_t dims[2] = {cuuint64_t(N), cuuint64_t(M)};
+  const cuuint64_t strides[1] = {cuuint64_t(ldy) * sizeof(__half)};
+  const cuuint32_t box[2] = {64, 32};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, Y, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+         CUDA_SUCCESS;
+}
+
 template <int BN>
 static int launch_tile(const CUtensorMap& ma, const CUtensorMap& mb, const Params& p, cudaStream_t st) {
   auto kern = w4a4_gemm_kernel<BN>;
@@ -874,16 +1255,18 @@ static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq,
   CUtensorMap ma, mb;
   if (pl.pair) {
     p.tiles_a = (p.rows_a + 255) / 256;
-    p.tiles_b = (p.rows_b + Pair::kBN - 1) / Pair::kBN;
-    if (!make_map(&ma, a_ptr, p.rows_a, K, kBM) || !make_map(&mb, b_ptr, p.rows_b, K, Pair::kHalfN))
+    p.tiles_b = (p.rows_b + PairT::kBN - 1) / PairT::kBN;
+    if (!make_map(&ma, a_ptr, p.rows_a, K, kBM) || !make_map(&mb, b_ptr, p.rows_b, K, PairT::kHalfN))
       return SMOOTHROT_CUDA_ERROR;
-    auto kern = w4a4_gemm_pair_kernel;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Pair::kSmemBytes) != cudaSuccess)
+    CUtensorMap my = ma;   // only read by the kernel when Y is written
+    if (p.Y != nullptr && !make_map_y(&my, p.Y, M, N, ldy)) return SMOOTHROT_CUDA_ERROR;
+    auto kern = w4a4_gemm_pair_tmem_kernel;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PairT::kSmemBytes) != cudaSuccess)
       return SMOOTHROT_CUDA_ERROR;
     const int total = p.tiles_a * p.tiles_b;
     const int pairs = sm_count() / 2;
     const int grid = 2 * (total < pairs ? total : pairs);
-    kern<<<grid, kThreads, Pair::kSmemBytes, st>>>(ma, mb, p);
+    kern<<<grid, kThreads, PairT::kSmemBytes, st>>>(ma, mb, my, p);
     count_launch();
     return launch_status();
   }
