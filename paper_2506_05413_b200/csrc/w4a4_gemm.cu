@@ -754,9 +754,10 @@ struct PairT {
   static constexpr int kWideB = kHalfN * kWideRow;
   static constexpr int kOutBoxBytes = 32 * 128;              // 32 rows x 64 fp16
   static constexpr int kOutBytes = kEpiWarps * 4 * kOutBoxBytes;  // 128 rows x 256 fp16
+  static constexpr int kDwBytes = kEpiWarps * kBN * 4;         // per epilogue warp: the tile's 256 weight steps
   static constexpr int kNumBarriers = 2 * kStages + 2 * kPackedStages + 2;
   static constexpr int kSmemBytes = 1024 + kStages * kWideB + kPackedStages * kPackedStageBytes + kOutBytes +
-                                    kNumBarriers * 8 + 16;
+                                    kDwBytes + kNumBarriers * 8 + 16;
   static constexpr int kTmemCols = 512;
   static constexpr int kAccCols = 256;
   static constexpr int kAWidenWarps = 4, kBWidenWarps = 4;
@@ -810,7 +811,8 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
   const uint32_t wide_base = base;                                             // int8 B stages
   const uint32_t packed_base = wide_base + T::kStages * T::kWideB;             // packed A + B stages
   const uint32_t out_base = packed_base + T::kPackedStages * T::kPackedStageBytes;  // fp16 output staging
-  const uint32_t bar_base = out_base + T::kOutBytes;
+  const uint32_t dw_base = out_base + T::kOutBytes;                            // weight steps of the current tile
+  const uint32_t bar_base = dw_base + T::kDwBytes;
   // full[s]: A slot s written in both CTAs' tensor memory and B stage s written in both CTAs' shared
   // memory (collected in the leader); empty[s]: the MMAs that read them have completed (both CTAs).
   auto full = [&](int s) { return bar_base + 8u * s; };
@@ -935,6 +937,9 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
             r[8 * c + 4 + i] = x[4 * c + i] & 0xF0F0F0F0u;
           }
         }
+        // the packed stage is in registers: give it back to the producer before waiting for a slot
+        __syncwarp();
+        if (lane == 0) mbar_arrive(pk_empty(ps));
         if (!mbar_wait(empty(s), sph ^ 1u, abort_flag, kSiteWidenEmpty)) { ok = false; break; }
         tcgen05_fence_after();
         tmem_store32(tmem_a_ring + (uint32_t(q * 32) << 16) + uint32_t(s * 32), r);
@@ -944,7 +949,6 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
         if (lane == 0) {
           if (leader) mbar_arrive(full(s));
           else mbar_arrive_cluster(map_to_cta(full(s), 0));
-          mbar_arrive(pk_empty(ps));
         }
       }
     }
@@ -963,32 +967,39 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
         const int s = it % T::kStages;
         const uint32_t sph = (it / T::kStages) & 1u;
         if (!mbar_wait(pk_full(ps), pph, abort_flag, kSiteWidenFull)) { ok = false; break; }
-        if (!mbar_wait(empty(s), sph ^ 1u, abort_flag, kSiteWidenEmpty)) { ok = false; break; }
         const uint32_t pk = packed_base + ps * T::kPackedStageBytes + T::kPackedA;
         const uint32_t wd = wide_base + s * T::kWideB;
+        constexpr int kPerWarp = kGroups / T::kBWidenWarps;
+        uint32_t x[kPerWarp][4];
 #pragma unroll
-        for (int g = w; g < kGroups; g += T::kBWidenWarps) {
-          const int row = g * 8 + r;
+        for (int u = 0; u < kPerWarp; ++u) {
+          const int row = (w + u * T::kBWidenWarps) * 8 + r;
           const uint32_t src = pk + row * kPackedRow + ((c ^ ((row >> 1) & 3)) << 4);
-          const uint32_t dst_row = wd + row * kWideRow;
-          uint32_t x0, x1, x2, x3;
           asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
-                       : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3) : "r"(src) : "memory");
+                       : "=r"(x[u][0]), "=r"(x[u][1]), "=r"(x[u][2]), "=r"(x[u][3]) : "r"(src) : "memory");
+        }
+        // the packed stage is in registers: give it back to the producer before waiting for a stage
+        __syncwarp();
+        if (lane == 0) mbar_arrive(pk_empty(ps));
+        if (!mbar_wait(empty(s), sph ^ 1u, abort_flag, kSiteWidenEmpty)) { ok = false; break; }
+#pragma unroll
+        for (int u = 0; u < kPerWarp; ++u) {
+          const int row = (w + u * T::kBWidenWarps) * 8 + r;
+          const uint32_t dst_row = wd + row * kWideRow;
           const uint32_t lo_dst = dst_row + (((2 * c) ^ (row & 7)) << 4);
           const uint32_t hi_dst = dst_row + (((2 * c + 1) ^ (row & 7)) << 4);
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                       ::"r"(lo_dst), "r"((x0 << 4) & 0xF0F0F0F0u), "r"((x1 << 4) & 0xF0F0F0F0u),
-                         "r"((x2 << 4) & 0xF0F0F0F0u), "r"((x3 << 4) & 0xF0F0F0F0u) : "memory");
+                       ::"r"(lo_dst), "r"((x[u][0] << 4) & 0xF0F0F0F0u), "r"((x[u][1] << 4) & 0xF0F0F0F0u),
+                         "r"((x[u][2] << 4) & 0xF0F0F0F0u), "r"((x[u][3] << 4) & 0xF0F0F0F0u) : "memory");
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                       ::"r"(hi_dst), "r"(x0 & 0xF0F0F0F0u), "r"(x1 & 0xF0F0F0F0u),
-                         "r"(x2 & 0xF0F0F0F0u), "r"(x3 & 0xF0F0F0F0u) : "memory");
+                       ::"r"(hi_dst), "r"(x[u][0] & 0xF0F0F0F0u), "r"(x[u][1] & 0xF0F0F0F0u),
+                         "r"(x[u][2] & 0xF0F0F0F0u), "r"(x[u][3] & 0xF0F0F0F0u) : "memory");
         }
         fence_proxy_async();
         __syncwarp();
         if (lane == 0) {
           if (leader) mbar_arrive(full(s));
           else mbar_arrive_cluster(map_to_cta(full(s), 0));
-          mbar_arrive(pk_empty(ps));
         }
       }
     }
@@ -997,19 +1008,35 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
     const int q = warp & 3;               // tensor-memory lane quadrant this warp may read
     const uint32_t out_warp = out_base + uint32_t(q) * uint32_t(4 * T::kOutBoxBytes);
     const uint32_t taddr = tmem_base + (uint32_t(q * 32) << 16);
+    const uint32_t dw_warp = dw_base + uint32_t(q) * uint32_t(T::kBN * 4);
     uint32_t local_tile = 0;
     for (int tile = first_tile; tile < total_tiles; tile += tile_step, ++local_tile) {
       const int ta = tile % p.tiles_a;
       const int tb = tile / p.tiles_a;
-      if (!mbar_wait(acc_full, local_tile & 1u, abort_flag, kSiteEpilogue)) break;
-      tcgen05_fence_after();
       const int row0 = ta * 256 + int(rank) * kBM + q * 32;
       const int a = row0 + lane;
+      float sx = 0.0f;
+      if (p.Y != nullptr) {
+        // fetch the scales while the tile is still being accumulated: this warp's copy of the
+        // tile's 256 weight steps goes to shared memory, the token step stays in a register
+        const int n = tb * T::kBN + lane * 8;
+        float4 w0 = make_float4(0.f, 0.f, 0.f, 0.f), w1 = w0;
+        if (n + 8 <= p.rows_b) {
+          w0 = __ldg(reinterpret_cast<const float4*>(p.dw + n));
+          w1 = __ldg(reinterpret_cast<const float4*>(p.dw + n + 4));
+        }
+        if (a < p.rows_a) sx = __ldg(p.dx + a) * 0.00390625f;   // accumulators are 256 * acc
+        float4* dst = reinterpret_cast<float4*>(smem + (dw_warp - base)) + lane * 2;
+        dst[0] = w0;
+        dst[1] = w1;
+        __syncwarp();
+      }
+      if (!mbar_wait(acc_full, local_tile & 1u, abort_flag, kSiteEpilogue)) break;
+      tcgen05_fence_after();
       if (p.Y != nullptr) {
         // the staging boxes of the previous tile must have been read by their TMA stores
         if (lane == 0) tma_store_wait_read();
         __syncwarp();
-        const float sx = a < p.rows_a ? __ldg(p.dx + a) * 0.00390625f : 0.0f;   // accumulators are 256 * acc
 #pragma unroll 1
         for (int cb = 0; cb < 4; ++cb) {
           const uint32_t box = out_warp + uint32_t(cb * T::kOutBoxBytes);
@@ -1027,15 +1054,11 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
                 else mbar_arrive_cluster(map_to_cta(acc_empty, 0));
               }
             }
-            const int n0 = tb * T::kBN + cb * 64 + h * 32;
+            const int n0 = cb * 64 + h * 32;   // column inside the tile
 #pragma unroll
             for (int jj = 0; jj < 4; ++jj) {
-              const int n = n0 + 8 * jj;
-              float4 w0 = make_float4(0.f, 0.f, 0.f, 0.f), w1 = w0;
-              if (n + 8 <= p.rows_b) {
-                w0 = __ldg(reinterpret_cast<const float4*>(p.dw + n));
-                w1 = __ldg(reinterpret_cast<const float4*>(p.dw + n + 4));
-              }
+              const float4* wsrc = reinterpret_cast<const float4*>(smem + (dw_warp - base)) + (n0 + 8 * jj) / 4;
+              const float4 w0 = wsrc[0], w1 = wsrc[1];
               const float ws[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
               uint32_t o[4];
 #pragma unroll
