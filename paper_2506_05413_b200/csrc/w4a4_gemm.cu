@@ -20,7 +20,9 @@
 //   scale and store, while the next tile's main loop runs on the other half
 //   of tensor memory.
 //
-// The kernel is persistent (one CTA per SM, tiles handed out round-robin).
+// The kernels are persistent (one CTA per SM, tiles handed out round-robin).
+// Shapes with M >= 256 and N >= 256 run the two-CTA kernel further down, which
+// keeps the token operand in tensor memory instead of shared memory.
 // For M < 128 tokens the roles of the operands are swapped (output channels on
 // the 128-row MMA axis, tokens on the N axis) and K is split across CTAs;
 // the int32 partial sums go to the caller's workspace and a second kernel
@@ -460,31 +462,16 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 // ---------------------------------------------------------------------------
 // Two-CTA kernel for prefill shapes.  A cluster of two CTAs (one SM pair)
 // computes one 256 x 256 output tile with tcgen05.mma.cta_group::2: each CTA
-// stages and widens its own 128 rows of the A side and HALF of the B side
-// (128 of the 256 output channels); the tensor cores of both SMs read the two
-// B halves, so per SM the widen work and the operand reads of B are halved.
+// holds its own 128 rows of the A side and stages HALF of the B side (128 of
+// the 256 output channels); the tensor cores of both SMs read the two B
+// halves, so per SM the widen work and the operand reads of B are halved.
 // The MMA is issued by one thread of the leader CTA (cluster rank 0).
 //
-// Barriers that collect arrivals from both CTAs (wide_full, acc_empty) live in
-// the leader; the peer's warps arrive on them through the cluster shared
-// window.  Barriers that release work in both CTAs (wide_empty, acc_full) are
-// signalled by tcgen05.commit with a two-CTA multicast mask.
+// Barriers that collect arrivals from both CTAs (full, acc_empty) live in the
+// leader; the peer's warps arrive on them through the cluster shared window.
+// Barriers that release work in both CTAs (empty, acc_full) are signalled by
+// tcgen05.commit with a two-CTA multicast mask.
 // ---------------------------------------------------------------------------
-struct Pair {
-  static constexpr int kBN = 256;     // output channels per pair tile
-  static constexpr int kHalfN = 128;  // B-side rows staged by each CTA
-  static constexpr int kWideStages = 3;
-  static constexpr int kPackedStages = 5;
-  static constexpr int kWideA = kBM * kWideRow, kWideB = kHalfN * kWideRow;
-  static constexpr int kPackedA = kBM * kPackedRow, kPackedB = kHalfN * kPackedRow;
-  static constexpr int kWideStageBytes = kWideA + kWideB;
-  static constexpr int kPackedStageBytes = kPackedA + kPackedB;
-  static constexpr int kNumBarriers = 2 * kWideStages + 2 * kPackedStages + 4;
-  static constexpr int kSmemBytes = 1024 + kWideStages * kWideStageBytes + kPackedStages * kPackedStageBytes +
-                                    kNumBarriers * 8 + 16;
-  static constexpr int kTmemCols = 512;  // two 256-column accumulators
-};
-
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
@@ -516,215 +503,13 @@ __device__ __forceinline__ void tcgen05_commit_pair(uint32_t bar) {
       ::"r"(bar), "h"(mask)
       : "memory");
 }
-__device__ __forceinline__ void mma_i8_pair(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
-                                            uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
 // int8 x int8 -> int32, K-major operands, M = 256 over the CTA pair.
 __host__ __device__ constexpr uint32_t make_idesc_i8_pair(int n) {
   return (2u << 4) | (1u << 7) | (1u << 10) | (uint32_t(n >> 3) << 17) | (uint32_t(256 >> 4) << 24);
 }
 
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
-w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                      const Params p) {
-  using T = Pair;
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t raw_addr = smem_u32(smem_raw);
-  const uint32_t base = (raw_addr + 1023u) & ~1023u;
-  uint8_t* smem = smem_raw + (base - raw_addr);
-
-  const uint32_t wide_base = base;
-  const uint32_t packed_base = wide_base + T::kWideStages * T::kWideStageBytes;
-  const uint32_t bar_base = packed_base + T::kPackedStages * T::kPackedStageBytes;
-  auto wide_full = [&](int s) { return bar_base + 8u * s; };
-  auto wide_empty = [&](int s) { return bar_base + 8u * (T::kWideStages + s); };
-  auto pk_full = [&](int s) { return bar_base + 8u * (2 * T::kWideStages + s); };
-  auto pk_empty = [&](int s) { return bar_base + 8u * (2 * T::kWideStages + T::kPackedStages + s); };
-  auto acc_full = [&](int s) { return bar_base + 8u * (2 * T::kWideStages + 2 * T::kPackedStages + s); };
-  auto acc_empty = [&](int s) { return bar_base + 8u * (2 * T::kWideStages + 2 * T::kPackedStages + 2 + s); };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + (bar_base - base) + 8 * T::kNumBarriers);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-
-  const int warp = threadIdx.x >> 5;
-  const int lane = threadIdx.x & 31;
-  const uint32_t rank = cluster_ctarank();
-  const bool leader = rank == 0;
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < T::kWideStages; ++s) {
-      mbar_init(wide_full(s), 2 * kWidenWarps);  // widen warps of both CTAs (used in the leader only)
-      mbar_init(wide_empty(s), 1);
-    }
-    for (int s = 0; s < T::kPackedStages; ++s) {
-      mbar_init(pk_full(s), 1);
-      mbar_init(pk_empty(s), kWidenWarps);
-    }
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(acc_full(s), 1);
-      mbar_init(acc_empty(s), 2 * kEpiWarps);    // epilogue warps of both CTAs (used in the leader only)
-    }
-    *abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    fence_proxy_async();
-  }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32(tmem_slot)), "r"(uint32_t(T::kTmemCols)) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-  }
-  tcgen05_fence_before();
-  __syncthreads();
-  cluster_sync_all();  // the peer's barriers exist before anyone arrives on them
-  tcgen05_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-
-  const int total_tiles = p.tiles_a * p.tiles_b;
-  const int first_tile = blockIdx.x >> 1;
-  const int tile_step = gridDim.x >> 1;
-  const int kblocks = p.kblocks;
-
-  if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer (each CTA, own data)
-    if (lane == 0) {
-      uint32_t it = 0;
-      bool ok = true;
-      for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
-        const int ta = tile % p.tiles_a;
-        const int tb = tile / p.tiles_a;
-        for (int kb = 0; kb < kblocks; ++kb, ++it) {
-          const int s = it % T::kPackedStages;
-          const uint32_t ph = (it / T::kPackedStages) & 1u;
-          if (!mbar_wait(pk_empty(s), ph ^ 1u, abort_flag, kSiteProducer)) { ok = false; break; }
-          mbar_expect_tx(pk_full(s), uint32_t(T::kPackedA + T::kPackedB));
-          const uint32_t dst = packed_base + s * T::kPackedStageBytes;
-          tma_load_2d(dst, &map_a, pk_full(s), kb * kPackedRow, ta * 256 + int(rank) * kBM);
-          tma_load_2d(dst + T::kPackedA, &map_b, pk_full(s), kb * kPackedRow, tb * T::kBN + int(rank) * T::kHalfN);
-        }
-      }
-    }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer (leader CTA only)
-    if (leader && lane == 0) {
-      constexpr uint32_t idesc = make_idesc_i8_pair(T::kBN);
-      uint32_t it = 0, local_tile = 0;
-      bool ok = true;
-      for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step, ++local_tile) {
-        const int ab = local_tile & 1;
-        const uint32_t aph = (local_tile >> 1) & 1u;
-        if (!mbar_wait(acc_empty(ab), aph ^ 1u, abort_flag, kSiteMmaAcc)) break;
-        tcgen05_fence_after();
-        const uint32_t tmem_d = tmem_base + uint32_t(ab * T::kBN);
-        for (int kb = 0; kb < kblocks; ++kb, ++it) {
-          const int s = it % T::kWideStages;
-          const uint32_t ph = (it / T::kWideStages) & 1u;
-          if (!mbar_wait(wide_full(s), ph, abort_flag, kSiteMmaWide)) { ok = false; break; }
-          tcgen05_fence_after();
-          const uint32_t a_addr = wide_base + s * T::kWideStageBytes;
-          const uint64_t da = make_desc_sw128(a_addr);
-          const uint64_t db = make_desc_sw128(a_addr + T::kWideA);
-#pragma unroll
-          for (int k4 = 0; k4 < 4; ++k4)
-            mma_i8_pair(tmem_d, da + uint64_t(2 * k4), db + uint64_t(2 * k4), idesc, (kb > 0 || k4 > 0) ? 1u : 0u);
-          tcgen05_commit_pair(wide_empty(s));
-        }
-        if (ok) tcgen05_commit_pair(acc_full(ab));
-      }
-    }
-  } else if (warp < 2 + kWidenWarps) {
-    // ------------------------------------------------------------ widen warps
-    const int w = warp - 2;
-    const int r = lane & 7;
-    const int c = lane >> 3;
-    constexpr int kGroupsA = kBM / 8;
-    constexpr int kGroups = (kBM + T::kHalfN) / 8;
-    uint32_t it = 0;
-    bool ok = true;
-    for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
-      for (int kb = 0; kb < kblocks; ++kb, ++it) {
-        const int ps = it % T::kPackedStages;
-        const uint32_t pph = (it / T::kPackedStages) & 1u;
-        const int ws = it % T::kWideStages;
-        const uint32_t wph = (it / T::kWideStages) & 1u;
-        if (!mbar_wait(pk_full(ps), pph, abort_flag, kSiteWidenFull)) { ok = false; break; }
-        if (!mbar_wait(wide_empty(ws), wph ^ 1u, abort_flag, kSiteWidenEmpty)) { ok = false; break; }
-        const uint32_t pk = packed_base + ps * T::kPackedStageBytes;
-        const uint32_t wd = wide_base + ws * T::kWideStageBytes;
-#pragma unroll
-        for (int g = w; g < kGroups; g += kWidenWarps) {
-          const bool is_b = g >= kGroupsA;
-          const int row = (is_b ? g - kGroupsA : g) * 8 + r;
-          const uint32_t src = (is_b ? pk + T::kPackedA : pk) + row * kPackedRow + ((c ^ ((row >> 1) & 3)) << 4);
-          const uint32_t dst_row = (is_b ? wd + T::kWideA : wd) + row * kWideRow;
-          uint32_t x0, x1, x2, x3;
-          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
-                       : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3) : "r"(src) : "memory");
-          const uint32_t lo_dst = dst_row + (((2 * c) ^ (row & 7)) << 4);
-          const uint32_t hi_dst = dst_row + (((2 * c + 1) ^ (row & 7)) << 4);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                       ::"r"(lo_dst), "r"((x0 << 4) & 0xF0F0F0F0u), "r"((x1 << 4) & 0xF0F0F0F0u),
-                         "r"((x2 << 4) & 0xF0F0F0F0u), "r"((x3 << 4) & 0xF0F0F0F0u) : "memory");
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                       ::"r"(hi_dst), "r"(x0 & 0xF0F0F0F0u), "r"(x1 & 0xF0F0F0F0u),
-                         "r"(x2 & 0xF0F0F0F0u), "r"(x3 & 0xF0F0F0F0u) : "memory");
-        }
-        fence_proxy_async();
-        __syncwarp();
-        if (lane == 0) {
-          if (leader) mbar_arrive(wide_full(ws));
-          else mbar_arrive_cluster(map_to_cta(wide_full(ws), 0));
-          mbar_arrive(pk_empty(ps));
-        }
-      }
-    }
-  } else {
-    // ------------------------------------------------------------ epilogue warps (each CTA, own 128 rows)
-    const int e = warp & 3;
-    uint32_t local_tile = 0;
-    for (int tile = first_tile; tile < total_tiles; tile += tile_step, ++local_tile) {
-      const int ta = tile % p.tiles_a;
-      const int tb = tile / p.tiles_a;
-      const int ab = local_tile & 1;
-      const uint32_t aph = (local_tile >> 1) & 1u;
-      if (!mbar_wait(acc_full(ab), aph, abort_flag, kSiteEpilogue)) break;
-      tcgen05_fence_after();
-      const int a = ta * 256 + int(rank) * kBM + e * 32 + lane;
-      const uint32_t taddr = tmem_base + (uint32_t(e * 32) << 16) + uint32_t(ab * T::kBN);
-#pragma unroll 1
-      for (int c0 = 0; c0 < T::kBN; c0 += 32) {
-        uint32_t regs[32];
-        tmem_load32(taddr + c0, regs);
-        tmem_wait_ld();
-        store_columns<32>(p, a, tb * T::kBN + c0, 0, regs);
-        __syncwarp();
-      }
-      tcgen05_fence_before();
-      __syncwarp();
-      if (lane == 0) {
-        if (leader) mbar_arrive(acc_empty(ab));
-        else mbar_arrive_cluster(map_to_cta(acc_empty(ab), 0));
-      }
-    }
-  }
-
-  tcgen05_fence_before();
-  __syncthreads();
-  cluster_sync_all();  // both CTAs are done with both halves of tensor memory
-  if (warp == 1) {
-    __syncwarp();
-    tcgen05_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;"
-                 ::"r"(tmem_base), "r"(uint32_t(T::kTmemCols)) : "memory");
-  }
-}
-
 // ---------------------------------------------------------------------------
-// Two-CTA kernel with the token operand in tensor memory.
+// The token operand lives in tensor memory.
 //
 // Shared-memory bandwidth (128 bytes per clock and SM, shared by TMA writes,
 // the widen warps and the tensor core's operand reads) is what bounds the
