@@ -44,6 +44,19 @@ inline bool split_order(int64_t K, int* base, int* n, int* logn) {
   return false;
 }
 
+// Number of SMs of the current device (148 on B200); cached after the first query.
+inline int device_sm_count() {
+  static std::atomic<int> cached{0};
+  int n = cached.load(std::memory_order_relaxed);
+  if (n > 0) return n;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+    return 148;
+  cached.store(n, std::memory_order_relaxed);
+  return n;
+}
+
 inline int launch_status() {
   return cudaGetLastError() == cudaSuccess ? SMOOTHROT_OK : SMOOTHROT_CUDA_ERROR;
 }

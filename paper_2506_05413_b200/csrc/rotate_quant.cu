@@ -213,23 +213,76 @@ rotate_generic_kernel(const __half* __restrict__ X, int64_t ldx, int K, int base
 }
 
 // ---------------------------------------------------------------------------
-// K = 4096.  A CTA holds kRowsPerCta rows, 64 threads (two warps) per row.
+// K = 4096.  Persistent kernel: one CTA per SM, kW4096Groups row groups of 64
+// threads (two warps) each; a group walks over rows  m, m + stride, ...
+//
+// The next row of a group is fetched by a bulk asynchronous copy
+// (cp.async.bulk, completion on an mbarrier) into the group's own 8 KB input
+// buffer while the current row is being transformed, so that the 8 groups of
+// an SM keep up to 64 KB of loads in flight and HBM never waits for arithmetic.
 //
 // Index bits of a row position j (12 bits):  i = j[0:3), t = j[3:9), g = j[9:12).
-//   phase 1  thread t loads the eight 16-byte chunks (g, t): values (g, i);
+//   phase 1  thread t reads the eight 16-byte chunks (g, t): values (g, i);
 //            butterflies on the bits of i and g (6 stages, in registers).
 //   transpose through shared memory: [t][g*8+i], row pitch 68 floats.
 //   phase 2  thread (g, i) holds the 64 values over t; butterflies on the six
-//            bits of t.  1/sqrt(4096) = 2^-6 is folded into `pre` (exact).
+//            bits of t.  1/sqrt(4096) = 2^-6 is folded into the step size (exact).
 //   absmax over the row, step size, rounding by the 1.5 * 2^23 trick, then the
 //   codes travel between the lanes of a row group so that each lane ends up
 //   with whole 32-bit words of packed output.
 // ---------------------------------------------------------------------------
-constexpr int kW4096Rows = 4;
+constexpr int kW4096Groups = 8;
+constexpr int kW4096Threads = kW4096Groups * 64;
 constexpr int kW4096Pitch = 68;  // floats per t-row in shared memory (64 + 4 pad)
+constexpr int kW4096PreBytes = 4096 * 4;
+constexpr int kW4096TileBytes = 64 * kW4096Pitch * 4;
+constexpr int kW4096InBytes = 4096 * 2;
+constexpr int kW4096GroupBytes = kW4096TileBytes + kW4096InBytes;
+constexpr int kW4096SmemBytes = kW4096PreBytes + kW4096Groups * kW4096GroupBytes + kW4096Groups * 8 + kW4096Groups * 4;
+constexpr unsigned long long kLoadWaitLimitNs = 2000000000ull;  // 2 s
+
+// Set when a bounded wait for a row copy ran out (read by smoothrot_device_status).
+__device__ int g_rotate_status = 0;
 
 __device__ __forceinline__ void group_barrier(int group) {
   asm volatile("bar.sync %0, 64;" ::"r"(group + 1) : "memory");
+}
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return uint32_t(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ bool row_copy_done(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+
+// Waits (bounded) until the bulk copy that was started on `bar` has landed.
+__device__ __forceinline__ bool wait_row_copy(uint32_t bar, uint32_t parity) {
+  if (row_copy_done(bar, parity)) return true;
+  unsigned long long t0;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+  for (uint32_t spin = 1;; ++spin) {
+    if (row_copy_done(bar, parity)) return true;
+    if ((spin & 255u) == 0u) {
+      unsigned long long now;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+      if (now - t0 > kLoadWaitLimitNs) {
+        atomicCAS(&g_rotate_status, 0, 16);
+        return false;
+      }
+    }
+  }
+}
+
+// Starts the copy of one row (bytes, a multiple of 16, both addresses 16-byte aligned).
+__device__ __forceinline__ void start_row_copy(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
 // Two fp32 values in one 64-bit register, for the packed add/sub/mul/fma of sm_100.
@@ -287,37 +340,71 @@ __device__ __forceinline__ void butterflies_pairs(f32x2* v) {
   }
 }
 
-// kLowClamp: whether codes below -8 can occur (only for clip ratios <= 7/8.5).
+// kLowClamp: the general two-sided clamp, needed when the row maximum can reach 8.5 steps or more
+// (clip ratios <= 7/8.5); otherwise only the code +8 can occur out of range and is fixed on the bytes.
 template <bool kQuant, bool kHasPre, bool kLowClamp>
-__global__ void __launch_bounds__(kW4096Rows * 64, 3)
+__global__ void __launch_bounds__(kW4096Threads, 1)
 walsh4096_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
                  const float* __restrict__ pre, float clip,
                  uint8_t* __restrict__ q_out, float* __restrict__ step_out,
                  float* __restrict__ y_out) {
-  extern __shared__ __align__(16) float smem[];
-  __shared__ float red[kW4096Rows][2];
+  // shared memory: [pre: 4096 fp32][per group: transpose tile | input row][per group: mbarrier][per group: flag]
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  __shared__ float red[kW4096Groups][2];
   const int group = threadIdx.x >> 6;
   const int t = threadIdx.x & 63;
   const int lane = threadIdx.x & 31;
-  const int64_t m = int64_t(blockIdx.x) * kW4096Rows + group;
-  if (m >= M) return;  // whole row group leaves together; only group barriers are used
-  float* tile = smem + group * (64 * kW4096Pitch);
+  float* spre = reinterpret_cast<float*>(smem_raw);
+  uint8_t* gbase = smem_raw + kW4096PreBytes + group * kW4096GroupBytes;
+  float* tile = reinterpret_cast<float*>(gbase);
+  const uint32_t inbuf = smem_addr(gbase + kW4096TileBytes);
+  const uint32_t bar = smem_addr(smem_raw + kW4096PreBytes + kW4096Groups * kW4096GroupBytes + group * 8);
+  volatile int* lost = reinterpret_cast<volatile int*>(smem_raw + kW4096PreBytes + kW4096Groups * kW4096GroupBytes +
+                                                         kW4096Groups * 8) + group;
+
+  if (kHasPre) {
+    for (int i = threadIdx.x; i < 1024; i += kW4096Threads)
+      reinterpret_cast<float4*>(spre)[i] = __ldg(reinterpret_cast<const float4*>(pre) + i);
+  }
+  if (t == 0) {
+    *lost = 0;
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  // rows of this group: blockIdx.x + gridDim.x * (group + kW4096Groups * k)
+  const int64_t stride = int64_t(gridDim.x) * kW4096Groups;
+  int64_t m = int64_t(blockIdx.x) + int64_t(gridDim.x) * group;
+  if (t == 0 && m < M) start_row_copy(inbuf, X + m * ldx, kW4096InBytes, bar);
+  uint32_t parity = 0;
+
+  for (; m < M; m += stride) {
+  // Every thread waits (bounded) for the row; a copy that never lands marks the group as lost and
+  // the group leaves together after its next barrier.
+  if (!wait_row_copy(bar, parity)) *lost = 1;
+  parity ^= 1u;
 
   // The values stay unnormalised until the end: 1/sqrt(4096) = 2^-6 is exact,
   // so it is folded into the step size (or applied at the fp32 store).
   f32x2 v[32];
   {
-    const __half* x = X + m * ldx;
     uint4 raw[8];
 #pragma unroll
-    for (int g = 0; g < 8; ++g) raw[g] = __ldg(reinterpret_cast<const uint4*>(x + g * 512 + t * 8));
+    for (int g = 0; g < 8; ++g)
+      asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                   : "=r"(raw[g].x), "=r"(raw[g].y), "=r"(raw[g].z), "=r"(raw[g].w)
+                   : "r"(inbuf + uint32_t(g * 1024 + t * 16)) : "memory");
+    group_barrier(group);   // the whole row is in registers: the buffer can take the next row
+    if (*lost != 0) break;
+    if (t == 0 && m + stride < M) start_row_copy(inbuf, X + (m + stride) * ldx, kW4096InBytes, bar);
 #pragma unroll
     for (int g = 0; g < 8; ++g) {
       const __half2* h = reinterpret_cast<const __half2*>(&raw[g]);
       float4 p0, p1;
       if (kHasPre) {
-        p0 = __ldg(reinterpret_cast<const float4*>(pre + g * 512 + t * 8));
-        p1 = __ldg(reinterpret_cast<const float4*>(pre + g * 512 + t * 8 + 4));
+        p0 = *reinterpret_cast<const float4*>(spre + g * 512 + t * 8);
+        p1 = *reinterpret_cast<const float4*>(spre + g * 512 + t * 8 + 4);
       }
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
@@ -361,7 +448,8 @@ walsh4096_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
       y[gi_g * 512 + (2 * u) * 8 + gi_i] = a * 0.015625f;
       y[gi_g * 512 + (2 * u + 1) * 8 + gi_i] = b * 0.015625f;
     }
-    return;
+    group_barrier(group);   // the tile is reused by the next row
+    continue;
   }
 
   float amax = 0.0f;
@@ -392,18 +480,20 @@ walsh4096_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
     for (int k = 0; k < 2; ++k) {
       float q0, q1;
       unpack2(fma2(v[2 * c + k], inv2, magic2), q0, q1);
-      q0 = fminf(q0, 12582912.0f + 15.0f);
-      q1 = fminf(q1, 12582912.0f + 15.0f);
       if (kLowClamp) {
-        q0 = fmaxf(q0, 12582912.0f);
-        q1 = fmaxf(q1, 12582912.0f);
+        q0 = fmaxf(fminf(q0, 12582912.0f + 15.0f), 12582912.0f);
+        q1 = fmaxf(fminf(q1, 12582912.0f + 15.0f), 12582912.0f);
       }
       r[2 * k] = __float_as_uint(q0);
       r[2 * k + 1] = __float_as_uint(q1);
     }
     const uint32_t lo = __byte_perm(r[0], r[1], 0x0040);  // bytes: r0.b0, r1.b0
     const uint32_t hi = __byte_perm(r[2], r[3], 0x0040);
-    spread[c] = __byte_perm(lo, hi, 0x5410);
+    uint32_t four = __byte_perm(lo, hi, 0x5410);
+    // Without the clamp above the row maximum sits below 8.5 steps, so a byte is code + 8 in
+    // [0, 16]; the one value out of range, 16 (code +8), comes down to 15: subtract bit 4 of each byte.
+    if (!kLowClamp) four -= (four >> 4) & 0x01010101u;
+    spread[c] = four;
   }
   // Lanes 2p and 2p+1 hold the even and odd position of each byte.  The even
   // lane finishes the words with even c, the odd lane those with odd c.
@@ -437,6 +527,7 @@ walsh4096_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
     const int u = 4 * (2 * c + (odd ? 1 : 0)) + r;
     q[gi_g * 64 + u] = w;
   }
+  }  // rows of this group
 }
 
 // ---------------------------------------------------------------------------
@@ -460,16 +551,15 @@ static int launch_rotate(const void* X, int64_t rows, int64_t K, int64_t ld, con
   if (rc != SMOOTHROT_OK || rows == 0) return rc;
   const __half* x = static_cast<const __half*>(X);
   if (K == 4096) {
-    const size_t smem = size_t(kW4096Rows) * 64 * kW4096Pitch * sizeof(float);
     // codes below -8 can only come up when the row maximum sits at 8.5 steps or more
     const bool low = kQuant && (7.0f / clip >= 8.49f);
     auto kern = pre ? (low ? walsh4096_kernel<kQuant, true, true> : walsh4096_kernel<kQuant, true, false>)
                     : (low ? walsh4096_kernel<kQuant, false, true> : walsh4096_kernel<kQuant, false, false>);
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess ||
-        cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, 100) != cudaSuccess)
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kW4096SmemBytes) != cudaSuccess)
       return SMOOTHROT_CUDA_ERROR;
-    const unsigned grid = unsigned((rows + kW4096Rows - 1) / kW4096Rows);
-    kern<<<grid, kW4096Rows * 64, smem, stream>>>(x, ld, rows, pre, clip, q_out, step_out, y_out);
+    const int sms = device_sm_count();
+    const unsigned grid = unsigned(rows < sms ? rows : sms);
+    kern<<<grid, kW4096Threads, kW4096SmemBytes, stream>>>(x, ld, rows, pre, clip, q_out, step_out, y_out);
     count_launch();
     return launch_status();
   }
@@ -513,6 +603,18 @@ int smoothrot_debug_hadamard(const void* X_f16, int64_t M, int64_t K, int64_t ld
   if (M > 0 && pre != nullptr && !smoothrot::aligned16(pre)) return SMOOTHROT_BAD_ALIGNMENT;
   return smoothrot::launch_rotate<false>(X_f16, M, K, ldx, pre, 1.0f, nullptr, nullptr, Y_f32,
                                          static_cast<cudaStream_t>(stream));
+}
+
+// Host. Timeout word of the row transform kernels on the current device (0 = none).
+int smoothrot_rotate_status_word(int* value, int clear) {
+  int v = 0;
+  if (cudaMemcpyFromSymbol(&v, smoothrot::g_rotate_status, sizeof(int)) != cudaSuccess) return SMOOTHROT_CUDA_ERROR;
+  *value = v;
+  if (clear && v != 0) {
+    const int zero = 0;
+    if (cudaMemcpyToSymbol(smoothrot::g_rotate_status, &zero, sizeof(int)) != cudaSuccess) return SMOOTHROT_CUDA_ERROR;
+  }
+  return SMOOTHROT_OK;
 }
 
 int smoothrot_paley28(int8_t* out_host) {

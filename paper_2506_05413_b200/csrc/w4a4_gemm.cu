@@ -35,6 +35,9 @@
 
 #include "common.cuh"
 
+// defined with the row transform kernels: their timeout word
+extern "C" int smoothrot_rotate_status_word(int* value, int clear);
+
 namespace smoothrot {
 namespace gemm {
 
@@ -1179,10 +1182,11 @@ int smoothrot_debug_gemm_i32(const uint8_t* Xq, int64_t M, const uint8_t* Wq, in
 
 int smoothrot_device_status(int* status_host, int clear) {
   if (status_host == nullptr) return SMOOTHROT_INVALID_ARG;
-  int v = 0;
+  int v = 0, rot = 0;
   if (cudaMemcpyFromSymbol(&v, smoothrot::gemm::g_device_status, sizeof(int)) != cudaSuccess)
     return SMOOTHROT_CUDA_ERROR;
-  *status_host = v;
+  if (smoothrot_rotate_status_word(&rot, clear) != SMOOTHROT_OK) return SMOOTHROT_CUDA_ERROR;
+  *status_host = v != 0 ? v : rot;
   if (clear && v != 0) {
     const int zero = 0;
     if (cudaMemcpyToSymbol(smoothrot::gemm::g_device_status, &zero, sizeof(int)) != cudaSuccess)
