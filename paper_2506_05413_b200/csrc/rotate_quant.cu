@@ -531,6 +531,298 @@ walsh4096_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
 }
 
 // ---------------------------------------------------------------------------
+// K = 14336 = 28 x 512  (index j = a * 512 + b; H = kron(H28, H512)).
+// Persistent kernel, one CTA per SM with kP512Groups row groups of 256 threads;
+// rows are prefetched by bulk asynchronous copies as in the K = 4096 kernel.
+//
+//   step 1  thread bp owns the two columns b = 2bp, 2bp + 1 and applies the
+//           order-28 factor to them: it reads the 28 fp16 pairs (a, b) from
+//           the input buffer four rows a at a time, multiplies by `pre`, and
+//           accumulates the 28 outputs.  Four inputs meet an output with one
+//           of 8 sign patterns (up to a global sign), so the 8 pattern sums
+//           are formed once per group of four (12 packed operations) and each
+//           output takes one add or subtract per group: about 4.5 packed
+//           operations per value instead of 13.5.
+//           The result goes to the fp32 row [28][512] in shared memory.
+//   step 2  thread (a, j), a < 28, j < 8, takes the eight 32-byte chunks
+//           j, j + 8, ... of row a: 64 values covering b bits {0,1,2} and
+//           {6,7,8}; six butterfly stages in registers, then the stages on b
+//           bits {3,4,5} across the 8 lanes j with warp shuffles.
+//   absmax over the row, step size, rounding; each chunk of 8 consecutive
+//   codes is one 32-bit word of output, assembled by its owner.
+// 1/sqrt(14336) is folded into the step size and the reciprocal.
+// ---------------------------------------------------------------------------
+constexpr int kP512Groups = 2;
+constexpr int kP512GroupThreads = 256;
+constexpr int kP512Threads = kP512Groups * kP512GroupThreads;
+constexpr int kP512K = 28 * 512;
+constexpr int kP512PreBytes = kP512K * 4;
+constexpr int kP512InBytes = kP512K * 2;
+constexpr int kP512RowBytes = kP512K * 4;
+constexpr int kP512GroupBytes = kP512InBytes + kP512RowBytes;
+constexpr int kP512SmemBytes = kP512PreBytes + kP512Groups * kP512GroupBytes + kP512Groups * 8 + kP512Groups * 4;
+static_assert(kP512SmemBytes <= 227 * 1024, "shared memory budget of the K = 14336 kernel");
+
+// For inputs 4g .. 4g+3 and output c: which of the 8 pattern sums, and whether it is added.
+// Pattern sums (first input always +):  0 ++++  1 ++--  2 +-+-  3 +--+  4 +++-  5 ++-+  6 +-++  7 +---
+struct Paley28Plan {
+  unsigned char index[7][28];
+  bool add[7][28];
+};
+
+__host__ __device__ constexpr Paley28Plan make_paley28_plan() {
+  Paley28Plan p{};
+  for (int g = 0; g < 7; ++g) {
+    for (int c = 0; c < 28; ++c) {
+      const int s0 = paley28_entry(4 * g, c), s1 = paley28_entry(4 * g + 1, c);
+      const int s2 = paley28_entry(4 * g + 2, c), s3 = paley28_entry(4 * g + 3, c);
+      // relative signs with respect to the first input
+      const int r1 = s1 * s0, r2 = s2 * s0, r3 = s3 * s0;
+      int idx = 0;
+      if (r1 > 0 && r2 > 0 && r3 > 0) idx = 0;
+      else if (r1 > 0 && r2 < 0 && r3 < 0) idx = 1;
+      else if (r1 < 0 && r2 > 0 && r3 < 0) idx = 2;
+      else if (r1 < 0 && r2 < 0 && r3 > 0) idx = 3;
+      else if (r1 > 0 && r2 > 0 && r3 < 0) idx = 4;
+      else if (r1 > 0 && r2 < 0 && r3 > 0) idx = 5;
+      else if (r1 < 0 && r2 > 0 && r3 > 0) idx = 6;
+      else idx = 7;
+      p.index[g][c] = static_cast<unsigned char>(idx);
+      p.add[g][c] = s0 > 0;
+    }
+  }
+  return p;
+}
+
+// Adds (or subtracts) the pattern sum the plan names for (group G, output C) to acc[C], for C = 0..27.
+template <int G, int C>
+struct Paley28Accumulate {
+  static __device__ __forceinline__ void run(f32x2* acc, const f32x2* sums) {
+    constexpr Paley28Plan plan = make_paley28_plan();
+    constexpr int idx = plan.index[G][C];
+    constexpr bool add = plan.add[G][C];
+    if (G == 0) {
+      static_assert(G != 0 || add, "the first row of the order-28 matrix is all +1");
+      acc[C] = sums[idx];
+    } else if (add) {
+      acc[C] = add2(acc[C], sums[idx]);
+    } else {
+      acc[C] = sub2(acc[C], sums[idx]);
+    }
+    if constexpr (C + 1 < 28) Paley28Accumulate<G, C + 1>::run(acc, sums);
+  }
+};
+
+// One group of four inputs (rows a = 4G .. 4G+3 of the order-28 factor) of step 1.
+template <int G, bool kHasPre>
+__device__ __forceinline__ void paley28_group(f32x2* acc, uint32_t in_addr, const float* spre, int bp) {
+  f32x2 x[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int a = 4 * G + q;
+    uint32_t raw;
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(raw) : "r"(in_addr + uint32_t(a * 1024 + bp * 4)) : "memory");
+    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&raw));
+    x[q] = pack2(f.x, f.y);
+    if (kHasPre) {
+      const float2 p = *reinterpret_cast<const float2*>(spre + a * 512 + bp * 2);
+      x[q] = mul2(x[q], pack2(p.x, p.y));
+    }
+  }
+  const f32x2 p0 = add2(x[0], x[1]), m0 = sub2(x[0], x[1]);
+  const f32x2 p1 = add2(x[2], x[3]), m1 = sub2(x[2], x[3]);
+  f32x2 sums[8];
+  sums[0] = add2(p0, p1);   // + + + +
+  sums[1] = sub2(p0, p1);   // + + - -
+  sums[2] = add2(m0, m1);   // + - + -
+  sums[3] = sub2(m0, m1);   // + - - +
+  sums[4] = add2(p0, m1);   // + + + -
+  sums[5] = sub2(p0, m1);   // + + - +
+  sums[6] = add2(m0, p1);   // + - + +
+  sums[7] = sub2(m0, p1);   // + - - -
+  Paley28Accumulate<G, 0>::run(acc, sums);
+}
+
+__device__ __forceinline__ void group_barrier256(int group) {
+  asm volatile("bar.sync %0, 256;" ::"r"(group + 1) : "memory");
+}
+
+template <bool kQuant, bool kHasPre, bool kLowClamp>
+__global__ void __launch_bounds__(kP512Threads, 1)
+paley512_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
+                const float* __restrict__ pre, float clip,
+                uint8_t* __restrict__ q_out, float* __restrict__ step_out,
+                float* __restrict__ y_out) {
+  // shared memory: [pre: 14336 fp32][per group: input row fp16 | transformed row fp32][mbarriers][flags]
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  __shared__ float red[kP512Groups][8];
+  const int group = threadIdx.x >> 8;
+  const int t = threadIdx.x & 255;
+  const int lane = threadIdx.x & 31;
+  float* spre = reinterpret_cast<float*>(smem_raw);
+  uint8_t* gbase = smem_raw + kP512PreBytes + group * kP512GroupBytes;
+  const uint32_t inbuf = smem_addr(gbase);
+  float* row = reinterpret_cast<float*>(gbase + kP512InBytes);
+  const uint32_t bar = smem_addr(smem_raw + kP512PreBytes + kP512Groups * kP512GroupBytes + group * 8);
+  volatile int* lost = reinterpret_cast<volatile int*>(smem_raw + kP512PreBytes + kP512Groups * kP512GroupBytes +
+                                                       kP512Groups * 8) + group;
+
+  if (kHasPre) {
+    for (int i = threadIdx.x; i < kP512K / 4; i += kP512Threads)
+      reinterpret_cast<float4*>(spre)[i] = __ldg(reinterpret_cast<const float4*>(pre) + i);
+  }
+  if (t == 0) {
+    *lost = 0;
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  const int64_t stride = int64_t(gridDim.x) * kP512Groups;
+  int64_t m = int64_t(blockIdx.x) + int64_t(gridDim.x) * group;
+  if (t == 0 && m < M) start_row_copy(inbuf, X + m * ldx, kP512InBytes, bar);
+  uint32_t parity = 0;
+
+  // step 2 ownership: row a of the order-28 factor, lane group j
+  const int a2 = t >> 3, j2 = t & 7;
+  const bool active2 = a2 < 28;
+
+  for (; m < M; m += stride) {
+    if (!wait_row_copy(bar, parity)) *lost = 1;
+    parity ^= 1u;
+
+    // ---- step 1: order-28 factor on columns 2t, 2t + 1 -------------------------------------
+    {
+      f32x2 acc[28];
+      paley28_group<0, kHasPre>(acc, inbuf, spre, t);
+      paley28_group<1, kHasPre>(acc, inbuf, spre, t);
+      paley28_group<2, kHasPre>(acc, inbuf, spre, t);
+      paley28_group<3, kHasPre>(acc, inbuf, spre, t);
+      paley28_group<4, kHasPre>(acc, inbuf, spre, t);
+      paley28_group<5, kHasPre>(acc, inbuf, spre, t);
+      paley28_group<6, kHasPre>(acc, inbuf, spre, t);
+      // fp32 row [28][512]; 16-byte units of a row are swapped in pairs where bit 3 of the unit
+      // index is set, which keeps step 2's 16-byte reads free of bank conflicts
+      const int unit = t >> 1;
+      const int phys = unit ^ ((unit >> 3) & 1);
+#pragma unroll
+      for (int c = 0; c < 28; ++c) {
+        float lo, hi;
+        unpack2(acc[c], lo, hi);
+        *reinterpret_cast<float2*>(row + c * 512 + phys * 4 + (t & 1) * 2) = make_float2(lo, hi);
+      }
+    }
+    group_barrier256(group);   // input consumed, transformed row complete
+    if (*lost != 0) break;
+    if (t == 0 && m + stride < M) start_row_copy(inbuf, X + (m + stride) * ldx, kP512InBytes, bar);
+
+    // ---- step 2: Walsh-512 along b ------------------------------------------------------------
+    f32x2 v[32];
+    if (active2) {
+      const int s = (j2 >> 2) & 1;   // the unit swap of this lane's chunks
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int chunk = j2 + 8 * k;                       // 8 consecutive b
+        const float4 h0 = *reinterpret_cast<const float4*>(row + a2 * 512 + (2 * chunk + s) * 4);
+        const float4 h1 = *reinterpret_cast<const float4*>(row + a2 * 512 + (2 * chunk + (s ^ 1)) * 4);
+        const float4 lo4 = h0, hi4 = h1;                    // logical order: b bits 0..2 = 0..3, 4..7
+        v[4 * k] = pack2(lo4.x, lo4.y);
+        v[4 * k + 1] = pack2(lo4.z, lo4.w);
+        v[4 * k + 2] = pack2(hi4.x, hi4.y);
+        v[4 * k + 3] = pack2(hi4.z, hi4.w);
+      }
+      butterflies_pairs<32>(v);   // b bits 0,1,2 (inside a chunk) and 6,7,8 (chunk index k)
+      // b bits 3,4,5 = lane bits 0,1,2: v' = partner + v on the lower lane, partner - v on the upper
+#pragma unroll
+      for (int bit = 1; bit < 8; bit <<= 1) {
+        const float sg = (j2 & bit) ? -1.0f : 1.0f;
+        const f32x2 sg2 = pack2(sg, sg);
+#pragma unroll
+        for (int u = 0; u < 32; ++u) {
+          float lo, hi;
+          unpack2(v[u], lo, hi);
+          const float plo = __shfl_xor_sync(0xffffffffu, lo, bit);
+          const float phi = __shfl_xor_sync(0xffffffffu, hi, bit);
+          v[u] = fma2(v[u], sg2, pack2(plo, phi));
+        }
+      }
+    }
+
+    const float isk = 0.00835190877f;   // 1 / sqrt(14336), rounded to fp32
+    if (!kQuant) {
+      if (active2) {
+        float* y = y_out + m * kP512K + a2 * 512;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          float4 o0, o1;
+          unpack2(v[4 * k], o0.x, o0.y);
+          unpack2(v[4 * k + 1], o0.z, o0.w);
+          unpack2(v[4 * k + 2], o1.x, o1.y);
+          unpack2(v[4 * k + 3], o1.z, o1.w);
+          o0.x *= isk; o0.y *= isk; o0.z *= isk; o0.w *= isk;
+          o1.x *= isk; o1.y *= isk; o1.z *= isk; o1.w *= isk;
+          float4* dst = reinterpret_cast<float4*>(y + (j2 + 8 * k) * 8);
+          dst[0] = o0;
+          dst[1] = o1;
+        }
+      }
+      group_barrier256(group);   // the row buffer is rewritten by the next row's step 1
+      continue;
+    }
+
+    float amax = 0.0f;
+    if (active2) {
+#pragma unroll
+      for (int u = 0; u < 32; ++u) {
+        float lo, hi;
+        unpack2(v[u], lo, hi);
+        amax = fmaxf(amax, fmaxf(fabsf(lo), fabsf(hi)));
+      }
+    }
+    amax = warp_max(amax);
+    if (lane == 0) red[group][t >> 5] = amax;
+    group_barrier256(group);
+    amax = red[group][0];
+#pragma unroll
+    for (int w = 1; w < 7; ++w) amax = fmaxf(amax, red[group][w]);
+    amax = __fmul_rn(amax, isk);                       // absmax of the normalised row
+    const float step = step_from_absmax(amax, clip);
+    if (t == 0) step_out[m] = step;
+    if (!active2) continue;
+    const float inv = __fmul_rn(__frcp_rn(step), isk);  // 1/step for the unnormalised values
+    const f32x2 inv2 = pack2(inv, inv);
+    const float kMagic = 12582912.0f + 8.0f;            // 1.5 * 2^23 + 8: low byte = code + 8
+    const f32x2 magic2 = pack2(kMagic, kMagic);
+    uint32_t* q = reinterpret_cast<uint32_t*>(q_out + m * (kP512K / 2)) + a2 * 64;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      uint32_t r[8];
+#pragma unroll
+      for (int p = 0; p < 4; ++p) {
+        float q0, q1;
+        unpack2(fma2(v[4 * k + p], inv2, magic2), q0, q1);
+        if (kLowClamp) {
+          q0 = fmaxf(fminf(q0, 12582912.0f + 15.0f), 12582912.0f);
+          q1 = fmaxf(fminf(q1, 12582912.0f + 15.0f), 12582912.0f);
+        }
+        r[2 * p] = __float_as_uint(q0);
+        r[2 * p + 1] = __float_as_uint(q1);
+      }
+      uint32_t lo4 = __byte_perm(__byte_perm(r[0], r[1], 0x0040), __byte_perm(r[2], r[3], 0x0040), 0x5410);
+      uint32_t hi4 = __byte_perm(__byte_perm(r[4], r[5], 0x0040), __byte_perm(r[6], r[7], 0x0040), 0x5410);
+      if (!kLowClamp) {   // bytes are code + 8 in [0, 16]: 16 comes down to 15
+        lo4 -= (lo4 >> 4) & 0x01010101u;
+        hi4 -= (hi4 >> 4) & 0x01010101u;
+      }
+      lo4 |= lo4 >> 4;    // bytes 0 and 2 now hold two codes each
+      hi4 |= hi4 >> 4;
+      const uint32_t word = __byte_perm(lo4, hi4, 0x6420) ^ 0x88888888u;   // offset binary -> two's complement
+      q[j2 + 8 * k] = word;
+    }
+  }  // rows of this group
+}
+
+// ---------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------
 static int check_rows(const void* X, int64_t rows, int64_t K, int64_t ld, int* base, int* n, int* logn) {
@@ -560,6 +852,18 @@ static int launch_rotate(const void* X, int64_t rows, int64_t K, int64_t ld, con
     const int sms = device_sm_count();
     const unsigned grid = unsigned(rows < sms ? rows : sms);
     kern<<<grid, kW4096Threads, kW4096SmemBytes, stream>>>(x, ld, rows, pre, clip, q_out, step_out, y_out);
+    count_launch();
+    return launch_status();
+  }
+  if (K == kP512K) {
+    const bool low = kQuant && (7.0f / clip >= 8.49f);
+    auto kern = pre ? (low ? paley512_kernel<kQuant, true, true> : paley512_kernel<kQuant, true, false>)
+                    : (low ? paley512_kernel<kQuant, false, true> : paley512_kernel<kQuant, false, false>);
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kP512SmemBytes) != cudaSuccess)
+      return SMOOTHROT_CUDA_ERROR;
+    const int sms = device_sm_count();
+    const unsigned grid = unsigned(rows < sms ? rows : sms);
+    kern<<<grid, kP512Threads, kP512SmemBytes, stream>>>(x, ld, rows, pre, clip, q_out, step_out, y_out);
     count_launch();
     return launch_status();
   }
