@@ -532,10 +532,10 @@ walsh4096_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
 
 // ---------------------------------------------------------------------------
 // K = 14336 = 28 x 512  (index j = a * 512 + b; H = kron(H28, H512)).
-// Persistent kernel, one CTA per SM with kP512Groups row groups of 256 threads;
+// Persistent kernel, one CTA per SM with kP512Groups row groups of 224 threads;
 // rows are prefetched by bulk asynchronous copies as in the K = 4096 kernel.
 //
-//   step 1  thread bp owns the two columns b = 2bp, 2bp + 1 and applies the
+//   step 1  a thread takes the two columns b = 2bp, 2bp + 1 and applies the
 //           order-28 factor to them: it reads the 28 fp16 pairs (a, b) from
 //           the input buffer four rows a at a time, multiplies by `pre`, and
 //           accumulates the 28 outputs.  Four inputs meet an output with one
@@ -546,14 +546,16 @@ walsh4096_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
 //           The result goes to the fp32 row [28][512] in shared memory.
 //   step 2  thread (a, j), a < 28, j < 8, takes the eight 32-byte chunks
 //           j, j + 8, ... of row a: 64 values covering b bits {0,1,2} and
-//           {6,7,8}; six butterfly stages in registers, then the stages on b
-//           bits {3,4,5} across the 8 lanes j with warp shuffles.
-//   absmax over the row, step size, rounding; each chunk of 8 consecutive
-//   codes is one 32-bit word of output, assembled by its owner.
+//           {6,7,8}; six butterfly stages in registers, results back in
+//           place; then the same 8 lanes re-read the row as 64 consecutive
+//           values each (chunks 8j .. 8j+7) and do the stages on b bits
+//           {3,4,5}, again in registers.
+//   absmax over the row, step size, rounding; a thread's 64 consecutive codes
+//   are eight 32-bit words of output, written as two 16-byte stores.
 // 1/sqrt(14336) is folded into the step size and the reciprocal.
 // ---------------------------------------------------------------------------
 constexpr int kP512Groups = 2;
-constexpr int kP512GroupThreads = 256;
+constexpr int kP512GroupThreads = 224;   // 28 rows a x 8 lanes: step 2 uses every thread
 constexpr int kP512Threads = kP512Groups * kP512GroupThreads;
 constexpr int kP512K = 28 * 512;
 constexpr int kP512PreBytes = kP512K * 4;
@@ -643,8 +645,13 @@ __device__ __forceinline__ void paley28_group(f32x2* acc, uint32_t in_addr, cons
   Paley28Accumulate<G, 0>::run(acc, sums);
 }
 
-__device__ __forceinline__ void group_barrier256(int group) {
-  asm volatile("bar.sync %0, 256;" ::"r"(group + 1) : "memory");
+// Position of 16-byte unit u (0..127) inside a 2 KB row of the fp32 buffer.  The low three bits
+// (the 128-byte bank group) are mixed with bits 3 and 4..6, so that 8 lanes reading units
+// 2 apart (step 2a), 16 apart (step 2b) or adjacent (step 1) never meet in a bank.
+__device__ __forceinline__ int p512_unit(int u) { return u ^ ((u >> 3) & 1) ^ ((u >> 4) & 7); }
+
+__device__ __forceinline__ void group_barrier224(int group) {
+  asm volatile("bar.sync %0, 224;" ::"r"(group + 1) : "memory");
 }
 
 template <bool kQuant, bool kHasPre, bool kLowClamp>
@@ -655,9 +662,9 @@ paley512_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
                 float* __restrict__ y_out) {
   // shared memory: [pre: 14336 fp32][per group: input row fp16 | transformed row fp32][mbarriers][flags]
   extern __shared__ __align__(128) uint8_t smem_raw[];
-  __shared__ float red[kP512Groups][8];
-  const int group = threadIdx.x >> 8;
-  const int t = threadIdx.x & 255;
+  __shared__ float red[kP512Groups][8];   // one slot per warp of a group (7 used)
+  const int group = threadIdx.x >= kP512GroupThreads ? 1 : 0;
+  const int t = threadIdx.x - group * kP512GroupThreads;
   const int lane = threadIdx.x & 31;
   float* spre = reinterpret_cast<float*>(smem_raw);
   uint8_t* gbase = smem_raw + kP512PreBytes + group * kP512GroupBytes;
@@ -685,72 +692,93 @@ paley512_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
 
   // step 2 ownership: row a of the order-28 factor, lane group j
   const int a2 = t >> 3, j2 = t & 7;
-  const bool active2 = a2 < 28;
 
   for (; m < M; m += stride) {
     if (!wait_row_copy(bar, parity)) *lost = 1;
     parity ^= 1u;
 
-    // ---- step 1: order-28 factor on columns 2t, 2t + 1 -------------------------------------
-    {
+    // ---- step 1: order-28 factor on a pair of columns; 256 pairs for 224 threads, so the
+    //      first warp of the group takes a second pair
+    for (int bp = t; bp < 256; bp += kP512GroupThreads) {
       f32x2 acc[28];
-      paley28_group<0, kHasPre>(acc, inbuf, spre, t);
-      paley28_group<1, kHasPre>(acc, inbuf, spre, t);
-      paley28_group<2, kHasPre>(acc, inbuf, spre, t);
-      paley28_group<3, kHasPre>(acc, inbuf, spre, t);
-      paley28_group<4, kHasPre>(acc, inbuf, spre, t);
-      paley28_group<5, kHasPre>(acc, inbuf, spre, t);
-      paley28_group<6, kHasPre>(acc, inbuf, spre, t);
-      // fp32 row [28][512]; 16-byte units of a row are swapped in pairs where bit 3 of the unit
-      // index is set, which keeps step 2's 16-byte reads free of bank conflicts
-      const int unit = t >> 1;
-      const int phys = unit ^ ((unit >> 3) & 1);
+      paley28_group<0, kHasPre>(acc, inbuf, spre, bp);
+      paley28_group<1, kHasPre>(acc, inbuf, spre, bp);
+      paley28_group<2, kHasPre>(acc, inbuf, spre, bp);
+      paley28_group<3, kHasPre>(acc, inbuf, spre, bp);
+      paley28_group<4, kHasPre>(acc, inbuf, spre, bp);
+      paley28_group<5, kHasPre>(acc, inbuf, spre, bp);
+      paley28_group<6, kHasPre>(acc, inbuf, spre, bp);
+      // fp32 row [28][512], its 16-byte units permuted by p512_unit
+      const int phys = p512_unit(bp >> 1);
 #pragma unroll
       for (int c = 0; c < 28; ++c) {
         float lo, hi;
         unpack2(acc[c], lo, hi);
-        *reinterpret_cast<float2*>(row + c * 512 + phys * 4 + (t & 1) * 2) = make_float2(lo, hi);
+        *reinterpret_cast<float2*>(row + c * 512 + phys * 4 + (bp & 1) * 2) = make_float2(lo, hi);
       }
     }
-    group_barrier256(group);   // input consumed, transformed row complete
+    group_barrier224(group);   // input consumed, transformed row complete
     if (*lost != 0) break;
     if (t == 0 && m + stride < M) start_row_copy(inbuf, X + (m + stride) * ldx, kP512InBytes, bar);
 
     // ---- step 2: Walsh-512 along b ------------------------------------------------------------
     f32x2 v[32];
-    if (active2) {
-      const int s = (j2 >> 2) & 1;   // the unit swap of this lane's chunks
+    {
+      float* arow = row + a2 * 512;
+      // 2a: chunks j, j + 8, ..: b bits 0,1,2 (inside a chunk) and 6,7,8 (k), in place
 #pragma unroll
       for (int k = 0; k < 8; ++k) {
-        const int chunk = j2 + 8 * k;                       // 8 consecutive b
-        const float4 h0 = *reinterpret_cast<const float4*>(row + a2 * 512 + (2 * chunk + s) * 4);
-        const float4 h1 = *reinterpret_cast<const float4*>(row + a2 * 512 + (2 * chunk + (s ^ 1)) * 4);
-        const float4 lo4 = h0, hi4 = h1;                    // logical order: b bits 0..2 = 0..3, 4..7
+        const int chunk = j2 + 8 * k;
+        const float4 lo4 = *reinterpret_cast<const float4*>(arow + p512_unit(2 * chunk) * 4);
+        const float4 hi4 = *reinterpret_cast<const float4*>(arow + p512_unit(2 * chunk + 1) * 4);
         v[4 * k] = pack2(lo4.x, lo4.y);
         v[4 * k + 1] = pack2(lo4.z, lo4.w);
         v[4 * k + 2] = pack2(hi4.x, hi4.y);
         v[4 * k + 3] = pack2(hi4.z, hi4.w);
       }
-      butterflies_pairs<32>(v);   // b bits 0,1,2 (inside a chunk) and 6,7,8 (chunk index k)
-      // b bits 3,4,5 = lane bits 0,1,2: v' = partner + v on the lower lane, partner - v on the upper
+      butterflies_pairs<32>(v);
 #pragma unroll
-      for (int bit = 1; bit < 8; bit <<= 1) {
-        const float sg = (j2 & bit) ? -1.0f : 1.0f;
-        const f32x2 sg2 = pack2(sg, sg);
+      for (int k = 0; k < 8; ++k) {
+        const int chunk = j2 + 8 * k;
+        float4 lo4, hi4;
+        unpack2(v[4 * k], lo4.x, lo4.y);
+        unpack2(v[4 * k + 1], lo4.z, lo4.w);
+        unpack2(v[4 * k + 2], hi4.x, hi4.y);
+        unpack2(v[4 * k + 3], hi4.z, hi4.w);
+        *reinterpret_cast<float4*>(arow + p512_unit(2 * chunk) * 4) = lo4;
+        *reinterpret_cast<float4*>(arow + p512_unit(2 * chunk + 1) * 4) = hi4;
+      }
+    }
+    __syncwarp();   // the 8 lanes that share row a sit in one warp
+    {
+      const float* arow = row + a2 * 512;
+      // 2b: the 8 consecutive chunks 8 j .. 8 j + 7 (64 consecutive b): b bits 3,4,5
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const int chunk = 8 * j2 + c;
+        const float4 lo4 = *reinterpret_cast<const float4*>(arow + p512_unit(2 * chunk) * 4);
+        const float4 hi4 = *reinterpret_cast<const float4*>(arow + p512_unit(2 * chunk + 1) * 4);
+        v[4 * c] = pack2(lo4.x, lo4.y);
+        v[4 * c + 1] = pack2(lo4.z, lo4.w);
+        v[4 * c + 2] = pack2(hi4.x, hi4.y);
+        v[4 * c + 3] = pack2(hi4.z, hi4.w);
+      }
+#pragma unroll
+      for (int h = 4; h < 32; h <<= 1) {   // pair index = 4 * c + p: the bits of c
 #pragma unroll
         for (int u = 0; u < 32; ++u) {
-          float lo, hi;
-          unpack2(v[u], lo, hi);
-          const float plo = __shfl_xor_sync(0xffffffffu, lo, bit);
-          const float phi = __shfl_xor_sync(0xffffffffu, hi, bit);
-          v[u] = fma2(v[u], sg2, pack2(plo, phi));
+          if ((u & h) == 0) {
+            const f32x2 x0 = v[u], x1 = v[u + h];
+            v[u] = add2(x0, x1);
+            v[u + h] = sub2(x0, x1);
+          }
         }
       }
     }
 
     const float isk = 0.00835190877f;   // 1 / sqrt(14336), rounded to fp32
     if (!kQuant) {
-      if (active2) {
+      {
         float* y = y_out + m * kP512K + a2 * 512;
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
@@ -761,17 +789,17 @@ paley512_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
           unpack2(v[4 * k + 3], o1.z, o1.w);
           o0.x *= isk; o0.y *= isk; o0.z *= isk; o0.w *= isk;
           o1.x *= isk; o1.y *= isk; o1.z *= isk; o1.w *= isk;
-          float4* dst = reinterpret_cast<float4*>(y + (j2 + 8 * k) * 8);
+          float4* dst = reinterpret_cast<float4*>(y + (8 * j2 + k) * 8);
           dst[0] = o0;
           dst[1] = o1;
         }
       }
-      group_barrier256(group);   // the row buffer is rewritten by the next row's step 1
+      group_barrier224(group);   // the row buffer is rewritten by the next row's step 1
       continue;
     }
 
     float amax = 0.0f;
-    if (active2) {
+    {
 #pragma unroll
       for (int u = 0; u < 32; ++u) {
         float lo, hi;
@@ -781,19 +809,19 @@ paley512_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
     }
     amax = warp_max(amax);
     if (lane == 0) red[group][t >> 5] = amax;
-    group_barrier256(group);
+    group_barrier224(group);
     amax = red[group][0];
 #pragma unroll
     for (int w = 1; w < 7; ++w) amax = fmaxf(amax, red[group][w]);
     amax = __fmul_rn(amax, isk);                       // absmax of the normalised row
     const float step = step_from_absmax(amax, clip);
     if (t == 0) step_out[m] = step;
-    if (!active2) continue;
     const float inv = __fmul_rn(__frcp_rn(step), isk);  // 1/step for the unnormalised values
     const f32x2 inv2 = pack2(inv, inv);
     const float kMagic = 12582912.0f + 8.0f;            // 1.5 * 2^23 + 8: low byte = code + 8
     const f32x2 magic2 = pack2(kMagic, kMagic);
     uint32_t* q = reinterpret_cast<uint32_t*>(q_out + m * (kP512K / 2)) + a2 * 64;
+    uint32_t words[8];
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
       uint32_t r[8];
@@ -817,8 +845,11 @@ paley512_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
       lo4 |= lo4 >> 4;    // bytes 0 and 2 now hold two codes each
       hi4 |= hi4 >> 4;
       const uint32_t word = __byte_perm(lo4, hi4, 0x6420) ^ 0x88888888u;   // offset binary -> two's complement
-      q[j2 + 8 * k] = word;
+      words[k] = word;
     }
+    uint4* dst = reinterpret_cast<uint4*>(q + 8 * j2);
+    dst[0] = make_uint4(words[0], words[1], words[2], words[3]);
+    dst[1] = make_uint4(words[4], words[5], words[6], words[7]);
   }  // rows of this group
 }
 
