@@ -564,6 +564,15 @@ __device__ __forceinline__ void mma_i8_pair_ts(uint32_t tmem_d, uint32_t tmem_a,
       : "memory");
 }
 
+// The odd codes of a packed word as int8 lanes (16 * code).  Volatile on purpose: the
+// instruction needs the loaded word, so the warp cannot go past it (to the arrival that hands the
+// packed stage back to the TMA producer) while the shared-memory load is still in flight.
+__device__ __forceinline__ uint32_t high_nibbles_now(uint32_t packed) {
+  uint32_t r;
+  asm volatile("and.b32 %0, %1, 0xF0F0F0F0;" : "=r"(r) : "r"(packed));
+  return r;
+}
+
 // 32 consecutive 32-bit columns of this thread's tensor-memory lane.
 __device__ __forceinline__ void tmem_store32(uint32_t taddr, const uint32_t* r) {
   asm volatile(
@@ -722,10 +731,11 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             r[8 * c + i] = (x[4 * c + i] << 4) & 0xF0F0F0F0u;
-            r[8 * c + 4 + i] = x[4 * c + i] & 0xF0F0F0F0u;
+            r[8 * c + 4 + i] = high_nibbles_now(x[4 * c + i]);
           }
         }
-        // the packed stage is in registers: give it back to the producer before waiting for a slot
+        // the packed stage is in registers (the instructions above have consumed every loaded
+        // word): give it back to the producer before waiting for a slot
         __syncwarp();
         if (lane == 0) mbar_arrive(pk_empty(ps));
         if (!mbar_wait(empty(s), sph ^ 1u, abort_flag, kSiteWidenEmpty)) { ok = false; break; }
@@ -766,7 +776,14 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
           asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
                        : "=r"(x[u][0]), "=r"(x[u][1]), "=r"(x[u][2]), "=r"(x[u][3]) : "r"(src) : "memory");
         }
-        // the packed stage is in registers: give it back to the producer before waiting for a stage
+        uint32_t hi[kPerWarp][4];
+#pragma unroll
+        for (int u = 0; u < kPerWarp; ++u) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) hi[u][i] = high_nibbles_now(x[u][i]);
+        }
+        // the packed stage is in registers (every loaded word has been consumed above): give it
+        // back to the producer before waiting for a stage
         __syncwarp();
         if (lane == 0) mbar_arrive(pk_empty(ps));
         if (!mbar_wait(empty(s), sph ^ 1u, abort_flag, kSiteWidenEmpty)) { ok = false; break; }
@@ -780,8 +797,7 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
                        ::"r"(lo_dst), "r"((x[u][0] << 4) & 0xF0F0F0F0u), "r"((x[u][1] << 4) & 0xF0F0F0F0u),
                          "r"((x[u][2] << 4) & 0xF0F0F0F0u), "r"((x[u][3] << 4) & 0xF0F0F0F0u) : "memory");
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                       ::"r"(hi_dst), "r"(x[u][0] & 0xF0F0F0F0u), "r"(x[u][1] & 0xF0F0F0F0u),
-                         "r"(x[u][2] & 0xF0F0F0F0u), "r"(x[u][3] & 0xF0F0F0F0u) : "memory");
+                       ::"r"(hi_dst), "r"(hi[u][0]), "r"(hi[u][1]), "r"(hi[u][2]), "r"(hi[u][3]) : "memory");
         }
         fence_proxy_async();
         __syncwarp();
