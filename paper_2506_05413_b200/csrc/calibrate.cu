@@ -118,7 +118,7 @@ static void launch_absmax(const __half* X, int64_t T, int64_t ldx, float* amax, 
                           int64_t ldw, float* wmax, int64_t K, cudaStream_t st) {
   const int64_t slabs = (K / 8 + kAbsmaxChunks - 1) / kAbsmaxChunks;
   const int64_t most_rows = T > N ? T : N;
-  int64_t row_sets = (int64_t(device_sm_count()) * kAbsmaxCtasPerSm + slabs - 1) / slabs;
+  int64_t row_sets = int64_t(device_sm_count()) * kAbsmaxCtasPerSm / slabs;   // rounded down: one wave, no tail
   const int64_t useful = (most_rows + kAbsmaxRowLanes - 1) / kAbsmaxRowLanes;   // beyond this, CTAs would idle
   if (row_sets > useful) row_sets = useful;
   if (row_sets < 1) row_sets = 1;

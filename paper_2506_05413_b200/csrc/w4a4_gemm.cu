@@ -548,10 +548,15 @@ struct PairT {
                                     kDwBytes + kNumBarriers * 8 + 16;
   static constexpr int kTmemCols = 512;
   static constexpr int kAccCols = 256;
-  static constexpr int kAWidenWarps = 4, kBWidenWarps = 4;
+  // Two sets of widen warps take the k-blocks in turn (even / odd), so that a warp has two
+  // k-block periods for its chain of waits, loads and stores; per k-block 4 A-widen warps (one
+  // per tensor-memory lane quadrant) and 4 B-widen warps are at work.
+  static constexpr int kWidenSets = 2;
+  static constexpr int kAWidenWarps = 4 * kWidenSets, kBWidenWarps = 4 * kWidenSets;
+  static constexpr int kArrivalsPerStage = 8;   // 4 A-widen + 4 B-widen warps per CTA and k-block
+  static constexpr int kThreads = 32 * (2 + kAWidenWarps + kBWidenWarps + kEpiWarps);
   static_assert(kAccCols + 32 * kStages <= kTmemCols, "A ring does not fit tensor memory");
   static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
-  static_assert(kAWidenWarps + kBWidenWarps == kWidenWarps, "warp roles");
 };
 
 __device__ __forceinline__ void mma_i8_pair_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc,
@@ -596,7 +601,7 @@ __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PairT::kThreads, 1)
 w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                            const __grid_constant__ CUtensorMap map_y, const Params p) {
   using T = PairT;
@@ -628,12 +633,12 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < T::kStages; ++s) {
-      mbar_init(full(s), 2 * kWidenWarps);   // A-widen and B-widen warps of both CTAs (used in the leader only)
+      mbar_init(full(s), 2 * T::kArrivalsPerStage);   // widen warps of both CTAs (used in the leader only)
       mbar_init(empty(s), 1);
     }
     for (int s = 0; s < T::kPackedStages; ++s) {
       mbar_init(pk_full(s), 1);
-      mbar_init(pk_empty(s), kWidenWarps);
+      mbar_init(pk_empty(s), T::kArrivalsPerStage);
     }
     mbar_init(acc_full, 1);
     mbar_init(acc_empty, 2 * kEpiWarps);     // epilogue warps of both CTAs (used in the leader only)
@@ -705,6 +710,7 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
   } else if (warp < 2 + T::kAWidenWarps) {
     // ------------------------------------------------------------ A-widen warps: packed rows -> tensor memory
     const int q = warp & 3;               // tensor-memory lane quadrant this warp may write
+    const uint32_t set = uint32_t(warp - 2) >> 2;   // which k-blocks this warp takes
     const int row = q * 32 + lane;        // A row inside the CTA's 128 = tensor-memory lane
     const uint32_t sw = uint32_t((row >> 1) & 3);
     uint32_t it = 0;
@@ -715,6 +721,7 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
         const uint32_t pph = (it / T::kPackedStages) & 1u;
         const int s = it % T::kStages;
         const uint32_t sph = (it / T::kStages) & 1u;
+        if ((it % T::kWidenSets) != set) continue;
         if (!mbar_wait(pk_full(ps), pph, abort_flag, kSiteWidenFull)) { ok = false; break; }
         const uint32_t src = packed_base + ps * T::kPackedStageBytes + row * kPackedRow;
         uint32_t x[16];
@@ -750,9 +757,10 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
         }
       }
     }
-  } else if (warp < 2 + kWidenWarps) {
+  } else if (warp < 2 + T::kAWidenWarps + T::kBWidenWarps) {
     // ------------------------------------------------------------ B-widen warps: packed rows -> int8 tile
-    const int w = warp - 2 - T::kAWidenWarps;
+    const int w = (warp - 2 - T::kAWidenWarps) & 3;
+    const uint32_t set = uint32_t(warp - 2 - T::kAWidenWarps) >> 2;   // which k-blocks this warp takes
     const int r = lane & 7;
     const int c = lane >> 3;
     constexpr int kGroups = T::kHalfN / 8;
@@ -764,14 +772,15 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
         const uint32_t pph = (it / T::kPackedStages) & 1u;
         const int s = it % T::kStages;
         const uint32_t sph = (it / T::kStages) & 1u;
+        if ((it % T::kWidenSets) != set) continue;
         if (!mbar_wait(pk_full(ps), pph, abort_flag, kSiteWidenFull)) { ok = false; break; }
         const uint32_t pk = packed_base + ps * T::kPackedStageBytes + T::kPackedA;
         const uint32_t wd = wide_base + s * T::kWideB;
-        constexpr int kPerWarp = kGroups / T::kBWidenWarps;
+        constexpr int kPerWarp = kGroups / 4;
         uint32_t x[kPerWarp][4];
 #pragma unroll
         for (int u = 0; u < kPerWarp; ++u) {
-          const int row = (w + u * T::kBWidenWarps) * 8 + r;
+          const int row = (w + u * 4) * 8 + r;
           const uint32_t src = pk + row * kPackedRow + ((c ^ ((row >> 1) & 3)) << 4);
           asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
                        : "=r"(x[u][0]), "=r"(x[u][1]), "=r"(x[u][2]), "=r"(x[u][3]) : "r"(src) : "memory");
@@ -789,7 +798,7 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
         if (!mbar_wait(empty(s), sph ^ 1u, abort_flag, kSiteWidenEmpty)) { ok = false; break; }
 #pragma unroll
         for (int u = 0; u < kPerWarp; ++u) {
-          const int row = (w + u * T::kBWidenWarps) * 8 + r;
+          const int row = (w + u * 4) * 8 + r;
           const uint32_t dst_row = wd + row * kWideRow;
           const uint32_t lo_dst = dst_row + (((2 * c) ^ (row & 7)) << 4);
           const uint32_t hi_dst = dst_row + (((2 * c + 1) ^ (row & 7)) << 4);
@@ -1093,7 +1102,7 @@ static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq,
     const int total = p.tiles_a * p.tiles_b;
     const int pairs = sm_count() / 2;
     const int grid = 2 * (total < pairs ? total : pairs);
-    kern<<<grid, kThreads, PairT::kSmemBytes, st>>>(ma, mb, my, p);
+    kern<<<grid, PairT::kThreads, PairT::kSmemBytes, st>>>(ma, mb, my, p);
     count_launch();
     return launch_status();
   }
