@@ -190,6 +190,7 @@ struct Params {
   int tiles_a, tiles_b;   // tile counts
   int kblocks;            // K / 128
   int splits;             // k-splits (1 = none)
+  int cluster_reduce;     // the k-splits of a tile form a thread-block cluster and add up in shared memory
   int swapped;            // 0: A side = tokens (Xq), B side = channels (Wq); 1: the reverse
   int M, N;               // logical output shape
   const float* dx;        // [M]
@@ -927,20 +928,364 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
   }
 }
 
-// Sums the split-K partials and applies the dequantization (or writes the int32 sum).
-__global__ void splitk_reduce_kernel(const int32_t* __restrict__ part, int splits, int M, int N,
-                                     const float* __restrict__ dx, const float* __restrict__ dw,
-                                     __half* __restrict__ Y, int64_t ldy, int32_t* __restrict__ acc_out) {
-  const int64_t idx = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
-  const int64_t total = int64_t(M) * N;
-  if (idx >= total) return;
-  int32_t sum = 0;
-  for (int s = 0; s < splits; ++s) sum += part[int64_t(s) * total + idx];
-  const int m = int(idx / N), n = int(idx % N);
-  if (Y != nullptr) {
-    Y[int64_t(m) * ldy + n] = __float2half_rn(float(sum) * (dx[m] * dw[n]));
+// ---------------------------------------------------------------------------
+// Weight-streaming kernel for M <= 128 tokens (decode and short prompts).
+//
+// The layer is then bound by the one pass over the packed weights, so the
+// kernel is built around that stream: output channels sit on the 128-row MMA
+// axis (operand A), the few tokens on the N axis (BN = 16 .. 128), K is split
+// across CTAs so that every SM streams.  As in the two-CTA kernel the streamed
+// operand never returns to shared memory: TMA delivers 64 packed bytes per
+// weight row and k-block, four A-widen warps (one per tensor-memory lane
+// quadrant) widen them in registers and tcgen05.st them into a ring of slots
+// in tensor memory, and the MMA takes A from there.  Only the token tile
+// (BN x 128 bytes per k-block) is widened into shared memory.  Per k-block a
+// CTA moves 16 KB of weight bytes through shared memory (TMA write + one read)
+// instead of 40 KB.  One CTA computes one (channel tile, k-split) and leaves;
+// two CTAs fit an SM (<= 256 tensor-memory columns each), which hides the fill
+// and drain of the short pipelines.  Partial sums of a split go to the
+// workspace as int32 and splitk_reduce_kernel adds them and dequantizes.
+// ---------------------------------------------------------------------------
+template <int BN>
+struct Stream {
+  static constexpr int kStages = BN <= 64 ? 6 : 4;       // A slots in tensor memory = token stages in shared memory
+  static constexpr int kPackedStages = 6;
+  static constexpr int kPackedA = kBM * kPackedRow;      // 8 KB of weights
+  static constexpr int kPackedB = BN * kPackedRow;
+  static constexpr int kPackedBPad = (kPackedB + 1023) / 1024 * 1024;
+  static constexpr int kPackedStageBytes = kPackedA + kPackedBPad;
+  static constexpr int kWideB = BN * kWideRow;
+  static constexpr int kWideBPad = (kWideB + 1023) / 1024 * 1024;
+  static constexpr int kAWidenWarps = 4, kBWidenWarps = BN >= 128 ? 4 : (BN >= 64 ? 2 : 1);
+  static constexpr int kArrivals = kAWidenWarps + kBWidenWarps;
+  static constexpr int kThreads = 32 * (2 + kAWidenWarps + kBWidenWarps + kEpiWarps);
+  static constexpr int kNumBarriers = 2 * kStages + 2 * kPackedStages + 1;
+  static constexpr int kSmemBytes = 1024 + kStages * kWideBPad + kPackedStages * kPackedStageBytes +
+                                    kNumBarriers * 8 + 16;
+  static constexpr int kTmemCols = 256;                  // accumulator (BN columns) + A ring (32 per slot)
+  static constexpr int kAccCols = BN;
+  static constexpr int kRingCol = BN <= 64 ? 64 : 128;   // the A ring starts here
+  static_assert(kRingCol + 32 * kStages <= kTmemCols && kAccCols <= kRingCol, "tensor-memory budget");
+};
+
+__device__ __forceinline__ void mma_i8_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+template <int BN>
+__global__ void __launch_bounds__(Stream<BN>::kThreads, BN >= 128 ? 1 : 2)
+w4a4_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                        const Params p) {
+  using T = Stream<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t base = (raw_addr + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - raw_addr);
+
+  const uint32_t wide_base = base;                                            // int8 token stages
+  const uint32_t packed_base = wide_base + T::kStages * T::kWideBPad;         // packed weights + tokens
+  const uint32_t bar_base = packed_base + T::kPackedStages * T::kPackedStageBytes;
+  auto full = [&](int s) { return bar_base + 8u * s; };
+  auto empty = [&](int s) { return bar_base + 8u * (T::kStages + s); };
+  auto pk_full = [&](int s) { return bar_base + 8u * (2 * T::kStages + s); };
+  auto pk_empty = [&](int s) { return bar_base + 8u * (2 * T::kStages + T::kPackedStages + s); };
+  const uint32_t acc_full = bar_base + 8u * (2 * T::kStages + 2 * T::kPackedStages);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + (bar_base - base) + 8 * T::kNumBarriers);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < T::kStages; ++s) {
+      mbar_init(full(s), T::kArrivals);
+      mbar_init(empty(s), 1);
+    }
+    for (int s = 0; s < T::kPackedStages; ++s) {
+      mbar_init(pk_full(s), 1);
+      mbar_init(pk_empty(s), T::kArrivals);
+    }
+    mbar_init(acc_full, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async();
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(tmem_slot)), "r"(uint32_t(T::kTmemCols)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_a_ring = tmem_base + uint32_t(T::kRingCol);
+
+  // this CTA's work: channel tile ta, token tile tb, k-split
+  // (the k-splits of a tile are neighbours in blockIdx.x, so that they can form a cluster)
+  const int split = blockIdx.x % p.splits;
+  const int tile = blockIdx.x / p.splits;
+  const int ta = tile % p.tiles_a;
+  const int tb = tile / p.tiles_a;
+  const int kb_count = p.kblocks / p.splits;   // host guarantees divisibility
+  const int kb0 = split * kb_count;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      for (int it = 0; it < kb_count; ++it) {
+        const int s = it % T::kPackedStages;
+        const uint32_t ph = uint32_t(it / T::kPackedStages) & 1u;
+        if (!mbar_wait(pk_empty(s), ph ^ 1u, abort_flag, kSiteProducer)) break;
+        mbar_expect_tx(pk_full(s), uint32_t(T::kPackedA + T::kPackedB));
+        const uint32_t dst = packed_base + s * T::kPackedStageBytes;
+        tma_load_2d(dst, &map_a, pk_full(s), (kb0 + it) * kPackedRow, ta * kBM);
+        tma_load_2d(dst + T::kPackedA, &map_b, pk_full(s), (kb0 + it) * kPackedRow, tb * BN);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_i8(BN);
+      bool ok = true;
+      for (int it = 0; it < kb_count; ++it) {
+        const int s = it % T::kStages;
+        const uint32_t ph = uint32_t(it / T::kStages) & 1u;
+        if (!mbar_wait(full(s), ph, abort_flag, kSiteMmaWide)) { ok = false; break; }
+        tcgen05_fence_after();
+        const uint64_t db = make_desc_sw128(wide_base + s * T::kWideBPad);
+        const uint32_t ta_addr = tmem_a_ring + uint32_t(s * 32);
+#pragma unroll
+        for (int k4 = 0; k4 < 4; ++k4)
+          mma_i8_ts(tmem_base, ta_addr + uint32_t(8 * k4), db + uint64_t(2 * k4), idesc, (it > 0 || k4 > 0) ? 1u : 0u);
+        tcgen05_commit(empty(s));
+      }
+      if (ok) tcgen05_commit(acc_full);
+    }
+  } else if (warp < 2 + T::kAWidenWarps) {
+    // ------------------------------------------------------------ A-widen warps: packed weight rows -> tensor memory
+    const int q = warp & 3;
+    const int row = q * 32 + lane;
+    const uint32_t sw = uint32_t((row >> 1) & 3);
+    for (int it = 0; it < kb_count; ++it) {
+      const int ps = it % T::kPackedStages;
+      const uint32_t pph = uint32_t(it / T::kPackedStages) & 1u;
+      const int s = it % T::kStages;
+      const uint32_t sph = uint32_t(it / T::kStages) & 1u;
+      if (!mbar_wait(pk_full(ps), pph, abort_flag, kSiteWidenFull)) break;
+      const uint32_t src = packed_base + ps * T::kPackedStageBytes + row * kPackedRow;
+      uint32_t x[16];
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(x[4 * c]), "=r"(x[4 * c + 1]), "=r"(x[4 * c + 2]), "=r"(x[4 * c + 3])
+                     : "r"(src + ((uint32_t(c) ^ sw) << 4)) : "memory");
+      uint32_t r[32];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          r[8 * c + i] = (x[4 * c + i] << 4) & 0xF0F0F0F0u;
+          r[8 * c + 4 + i] = high_nibbles_now(x[4 * c + i]);
+        }
+      }
+      // every loaded word has been consumed: the packed stage can go back to the producer
+      __syncwarp();
+      if (lane == 0) mbar_arrive(pk_empty(ps));
+      if (!mbar_wait(empty(s), sph ^ 1u, abort_flag, kSiteWidenEmpty)) break;
+      tcgen05_fence_after();
+      tmem_store32(tmem_a_ring + (uint32_t(q * 32) << 16) + uint32_t(s * 32), r);
+      tmem_wait_st();
+      tcgen05_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(full(s));
+    }
+  } else if (warp < 2 + T::kAWidenWarps + T::kBWidenWarps) {
+    // ------------------------------------------------------------ B-widen warps: packed token rows -> int8 tile
+    const int w = warp - 2 - T::kAWidenWarps;
+    const int r = lane & 7;
+    const int c = lane >> 3;
+    constexpr int kGroups = BN / 8;
+    for (int it = 0; it < kb_count; ++it) {
+      const int ps = it % T::kPackedStages;
+      const uint32_t pph = uint32_t(it / T::kPackedStages) & 1u;
+      const int s = it % T::kStages;
+      const uint32_t sph = uint32_t(it / T::kStages) & 1u;
+      if (!mbar_wait(pk_full(ps), pph, abort_flag, kSiteWidenFull)) break;
+      if (!mbar_wait(empty(s), sph ^ 1u, abort_flag, kSiteWidenEmpty)) break;
+      const uint32_t pk = packed_base + ps * T::kPackedStageBytes + T::kPackedA;
+      const uint32_t wd = wide_base + s * T::kWideBPad;
+#pragma unroll
+      for (int g = w; g < kGroups; g += T::kBWidenWarps) {
+        const int row = g * 8 + r;
+        const uint32_t src = pk + row * kPackedRow + ((c ^ ((row >> 1) & 3)) << 4);
+        const uint32_t dst_row = wd + row * kWideRow;
+        uint32_t x0, x1, x2, x3;
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3) : "r"(src) : "memory");
+        const uint32_t lo_dst = dst_row + (((2 * c) ^ (row & 7)) << 4);
+        const uint32_t hi_dst = dst_row + (((2 * c + 1) ^ (row & 7)) << 4);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                     ::"r"(lo_dst), "r"((x0 << 4) & 0xF0F0F0F0u), "r"((x1 << 4) & 0xF0F0F0F0u),
+                       "r"((x2 << 4) & 0xF0F0F0F0u), "r"((x3 << 4) & 0xF0F0F0F0u) : "memory");
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                     ::"r"(hi_dst), "r"(x0 & 0xF0F0F0F0u), "r"(x1 & 0xF0F0F0F0u),
+                       "r"(x2 & 0xF0F0F0F0u), "r"(x3 & 0xF0F0F0F0u) : "memory");
+      }
+      // the stores above consumed the loaded words, so the packed stage is free as well
+      fence_proxy_async();
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(full(s));
+        mbar_arrive(pk_empty(ps));
+      }
+    }
   } else {
-    acc_out[idx] = sum;
+    // ------------------------------------------------------------ epilogue warps
+    const int e = warp & 3;
+    if (mbar_wait(acc_full, 0u, abort_flag, kSiteEpilogue)) {
+      tcgen05_fence_after();
+      const int a = ta * kBM + e * 32 + lane;
+      const uint32_t taddr = tmem_base + (uint32_t(e * 32) << 16);
+      if (p.cluster_reduce) {
+        // this split's partial sums, token-major [BN][128] int32, over the int8 token stages
+        // (every MMA that read them has completed)
+        const uint32_t dst = wide_base + uint32_t(e * 32 + lane) * 4u;
+        if constexpr (BN >= 32) {
+#pragma unroll 1
+          for (int c0 = 0; c0 < BN; c0 += 32) {
+            uint32_t regs[32];
+            tmem_load32(taddr + uint32_t(c0), regs);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              asm volatile("st.shared.b32 [%0], %1;" ::"r"(dst + uint32_t(c0 + j) * 512u), "r"(regs[j]) : "memory");
+          }
+        } else {
+          uint32_t regs[16];
+          tmem_load16(taddr, regs);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            asm volatile("st.shared.b32 [%0], %1;" ::"r"(dst + uint32_t(j) * 512u), "r"(regs[j]) : "memory");
+        }
+      } else if constexpr (BN >= 32) {
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          uint32_t regs[32];
+          tmem_load32(taddr + uint32_t(c0), regs);
+          tmem_wait_ld();
+          store_columns<32>(p, a, tb * BN + c0, split, regs);
+          __syncwarp();
+        }
+      } else {
+        uint32_t regs[16];
+        tmem_load16(taddr, regs);
+        tmem_wait_ld();
+        store_columns<16>(p, a, tb * BN, split, regs);
+        __syncwarp();
+      }
+    }
+  }
+
+  tcgen05_fence_before();
+  __syncthreads();
+  if (p.cluster_reduce) {
+    // The CTAs of a cluster hold the partial sums of one tile for their k-splits.  Each CTA
+    // adds up a slice of 128 / splits channels over all of them, read through the cluster's
+    // shared-memory window, and writes the finished outputs.
+    cluster_sync_all();
+    const int slice = kBM / p.splits;              // 16, 32 or 64 channels
+    const int tokens = min(BN, p.rows_b - tb * BN);
+    const int n_local0 = split * slice;
+    const int quads = slice / 4;                   // a thread adds up 4 consecutive channels of one token
+    for (int idx = threadIdx.x; idx < tokens * quads; idx += T::kThreads) {
+      const int mi = idx / quads;                  // token inside the tile
+      const int nl = n_local0 + (idx % quads) * 4; // first channel inside the tile
+      const uint32_t off = wide_base + uint32_t(mi * kBM + nl) * 4u;
+      int4 part[8];
+#pragma unroll
+      for (int r = 0; r < 8; ++r) {
+        part[r] = make_int4(0, 0, 0, 0);
+        if (r < p.splits)
+          asm volatile("ld.shared::cluster.v4.b32 {%0, %1, %2, %3}, [%4];"
+                       : "=r"(part[r].x), "=r"(part[r].y), "=r"(part[r].z), "=r"(part[r].w)
+                       : "r"(map_to_cta(off, uint32_t(r))) : "memory");
+      }
+      int sum[4] = {0, 0, 0, 0};
+#pragma unroll
+      for (int r = 0; r < 8; ++r) {
+        sum[0] += part[r].x; sum[1] += part[r].y; sum[2] += part[r].z; sum[3] += part[r].w;
+      }
+      const int n = ta * kBM + nl;
+      const int m = tb * BN + mi;
+      if (n < p.rows_a) {                          // channel counts are multiples of 8: all four or none
+        if (p.Y != nullptr) {
+          const float sx = __ldg(p.dx + m);
+          const float4 sw = __ldg(reinterpret_cast<const float4*>(p.dw + n));
+          const __half2 h0 = __floats2half2_rn(float(sum[0] >> 8) * (sx * sw.x), float(sum[1] >> 8) * (sx * sw.y));
+          const __half2 h1 = __floats2half2_rn(float(sum[2] >> 8) * (sx * sw.z), float(sum[3] >> 8) * (sx * sw.w));
+          uint2 out;
+          out.x = *reinterpret_cast<const uint32_t*>(&h0);
+          out.y = *reinterpret_cast<const uint32_t*>(&h1);
+          *reinterpret_cast<uint2*>(p.Y + int64_t(m) * p.ldy + n) = out;
+        } else {
+          *reinterpret_cast<int4*>(p.acc_out + int64_t(m) * p.N + n) =
+              make_int4(sum[0] >> 8, sum[1] >> 8, sum[2] >> 8, sum[3] >> 8);
+        }
+      }
+    }
+    cluster_sync_all();   // nobody leaves while its shared memory may still be read
+  }
+  if (warp == 1) {
+    __syncwarp();
+    tcgen05_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
+                 ::"r"(tmem_base), "r"(uint32_t(T::kTmemCols)) : "memory");
+  }
+}
+
+// Sums the split-K partials and applies the dequantization (or writes the int32 sum).
+// A thread owns 8 consecutive output channels of one token (N is a multiple of 8).
+__global__ void __launch_bounds__(256)
+splitk_reduce_kernel(const int32_t* __restrict__ part, int splits, int M, int N,
+                     const float* __restrict__ dx, const float* __restrict__ dw,
+                     __half* __restrict__ Y, int64_t ldy, int32_t* __restrict__ acc_out) {
+  const int n8 = N >> 3;
+  const int64_t idx = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= int64_t(M) * n8) return;
+  const int m = int(idx / n8);
+  const int n = int(idx - int64_t(m) * n8) * 8;
+  const int64_t plane = int64_t(M) * N;
+  const int4* src = reinterpret_cast<const int4*>(part + int64_t(m) * N + n);
+  int4 s0 = make_int4(0, 0, 0, 0), s1 = s0;
+  for (int s = 0; s < splits; ++s) {
+    const int4 a = __ldcs(src), b = __ldcs(src + 1);   // read once: keep the partials out of the way in L2
+    s0.x += a.x; s0.y += a.y; s0.z += a.z; s0.w += a.w;
+    s1.x += b.x; s1.y += b.y; s1.z += b.z; s1.w += b.w;
+    src += plane / 4;
+  }
+  if (Y != nullptr) {
+    const float sx = __ldg(dx + m);
+    const float4 w0 = __ldg(reinterpret_cast<const float4*>(dw + n));
+    const float4 w1 = __ldg(reinterpret_cast<const float4*>(dw + n + 4));
+    uint4 out;
+    __half2* h = reinterpret_cast<__half2*>(&out);
+    h[0] = __floats2half2_rn(float(s0.x) * (sx * w0.x), float(s0.y) * (sx * w0.y));
+    h[1] = __floats2half2_rn(float(s0.z) * (sx * w0.z), float(s0.w) * (sx * w0.w));
+    h[2] = __floats2half2_rn(float(s1.x) * (sx * w1.x), float(s1.y) * (sx * w1.y));
+    h[3] = __floats2half2_rn(float(s1.z) * (sx * w1.z), float(s1.w) * (sx * w1.w));
+    *reinterpret_cast<uint4*>(Y + int64_t(m) * ldy + n) = out;
+  } else {
+    int4* o = reinterpret_cast<int4*>(acc_out + int64_t(m) * N + n);
+    o[0] = s0;
+    o[1] = s1;
   }
 }
 
@@ -949,7 +1294,8 @@ __global__ void splitk_reduce_kernel(const int32_t* __restrict__ part, int split
 // ---------------------------------------------------------------------------
 struct Plan {
   bool swapped;
-  bool pair;   // two-CTA kernel, 256 x 256 pair tiles
+  bool pair;      // two-CTA kernel, 256 x 256 pair tiles
+  bool cluster;   // the k-splits of a tile form a cluster and add up in shared memory (no workspace)
   int bn;
   int splits;
 };
@@ -970,7 +1316,7 @@ static int sm_count() {
 static Plan make_plan(int64_t M, int64_t N, int64_t K) {
   Plan pl{};
   const int kblocks = int(K / kWideRow);
-  if (M >= 128) {
+  if (M > 128) {
     pl.swapped = false;
     pl.pair = M >= 256 && N >= 256;
     pl.bn = (N >= 256) ? 256 : (N > 64 ? 128 : 64);
@@ -980,12 +1326,26 @@ static Plan make_plan(int64_t M, int64_t N, int64_t K) {
   pl.swapped = true;
   pl.bn = M <= 16 ? 16 : (M <= 32 ? 32 : (M <= 64 ? 64 : 128));
   const int tiles = int((N + kBM - 1) / kBM);
-  int want = (sm_count() + tiles - 1) / tiles;
+  // two CTAs of the streaming kernel share an SM, except with the 128-token tile
+  const int slots = (pl.bn <= 64 ? 2 : 1) * sm_count();
+  int want = (slots + tiles - 1) / tiles;
   if (want < 1) want = 1;
-  int splits = 1;
-  // largest divisor of kblocks that does not exceed `want` and leaves >= 4 k-blocks per split
+  // Workspace path: the largest divisor of kblocks that does not exceed `want` and leaves >= 4
+  // k-blocks per split.  Cluster path: the same among 1, 2, 4, 8 (portable cluster sizes that
+  // divide the 128 channels of a tile).  The cluster path needs no workspace and no second
+  // kernel, so it is taken unless the workspace path offers at least four times the CTAs while
+  // the cluster path would leave more than half of the machine idle.
+  int splits = 1, csplits = 1;
   for (int s = 1; s <= kblocks && s <= want; ++s)
     if (kblocks % s == 0 && kblocks / s >= 4) splits = s;
+  for (int s = 1; s <= 8 && s <= want; s *= 2)
+    if (kblocks % s == 0 && kblocks / s >= 4) csplits = s;
+  if (splits >= 4 * csplits && 2 * csplits * tiles < slots) {
+    pl.cluster = false;
+  } else {
+    pl.cluster = csplits > 1;
+    splits = csplits;
+  }
   pl.splits = splits;
   return pl;
 }
@@ -1033,6 +1393,37 @@ static bool make_map_y(CUtensorMap* map, __half* Y, int64_t M, int64_t N, int64_
 }
 
 template <int BN>
+static int launch_stream(const CUtensorMap& ma, const CUtensorMap& mb, const Params& p, cudaStream_t st) {
+  auto kern = w4a4_gemm_stream_kernel<BN>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Stream<BN>::kSmemBytes) != cudaSuccess)
+    return SMOOTHROT_CUDA_ERROR;
+  const int total = p.tiles_a * p.tiles_b * p.splits;   // one CTA per (channel tile, token tile, k-split)
+  if (p.cluster_reduce) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(unsigned(total), 1, 1);
+    cfg.blockDim = dim3(unsigned(Stream<BN>::kThreads), 1, 1);
+    cfg.dynamicSmemBytes = size_t(Stream<BN>::kSmemBytes);
+    cfg.stream = st;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = unsigned(p.splits);
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kern, ma, mb, p) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return SMOOTHROT_CUDA_ERROR;
+    }
+    count_launch();
+    return launch_status();
+  }
+  kern<<<total, Stream<BN>::kThreads, Stream<BN>::kSmemBytes, st>>>(ma, mb, p);
+  count_launch();
+  return launch_status();
+}
+
+template <int BN>
 static int launch_tile(const CUtensorMap& ma, const CUtensorMap& mb, const Params& p, cudaStream_t st) {
   auto kern = w4a4_gemm_kernel<BN>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Tile<BN>::kSmemBytes) != cudaSuccess)
@@ -1062,7 +1453,7 @@ static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq,
     if (!aligned16(acc_out)) return SMOOTHROT_BAD_ALIGNMENT;
   }
   const Plan pl = make_plan(M, N, K);
-  const size_t need = pl.splits > 1 ? size_t(pl.splits) * size_t(M) * size_t(N) * sizeof(int32_t) : 0;
+  const size_t need = (pl.splits > 1 && !pl.cluster) ? size_t(pl.splits) * size_t(M) * size_t(N) * sizeof(int32_t) : 0;
   if (need > 0 && (workspace == nullptr || workspace_bytes < need)) return SMOOTHROT_WORKSPACE_TOO_SMALL;
   if (need > 0 && !aligned16(workspace)) return SMOOTHROT_BAD_ALIGNMENT;
 
@@ -1076,12 +1467,13 @@ static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq,
   p.tiles_b = (p.rows_b + pl.bn - 1) / pl.bn;
   p.kblocks = int(K / kWideRow);
   p.splits = pl.splits;
+  p.cluster_reduce = pl.cluster ? 1 : 0;
   p.M = int(M);
   p.N = int(N);
   p.dx = dx;
   p.dw = dw;
   p.ldy = ldy;
-  if (pl.splits > 1) {
+  if (pl.splits > 1 && !pl.cluster) {
     p.Y = nullptr;
     p.acc_out = static_cast<int32_t*>(workspace);
   } else {
@@ -1109,6 +1501,14 @@ static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq,
   if (!make_map(&ma, a_ptr, p.rows_a, K, kBM) || !make_map(&mb, b_ptr, p.rows_b, K, pl.bn))
     return SMOOTHROT_CUDA_ERROR;
   int rc;
+  if (pl.swapped) {
+    switch (pl.bn) {
+      case 128: rc = launch_stream<128>(ma, mb, p, st); break;
+      case 64: rc = launch_stream<64>(ma, mb, p, st); break;
+      case 32: rc = launch_stream<32>(ma, mb, p, st); break;
+      default: rc = launch_stream<16>(ma, mb, p, st); break;
+    }
+  } else
   switch (pl.bn) {
     case 256: rc = launch_tile<256>(ma, mb, p, st); break;
     case 128: rc = launch_tile<128>(ma, mb, p, st); break;
@@ -1117,8 +1517,8 @@ static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq,
     default: rc = launch_tile<16>(ma, mb, p, st); break;
   }
   if (rc != SMOOTHROT_OK) return rc;
-  if (pl.splits > 1) {
-    const int64_t total = M * N;
+  if (pl.splits > 1 && !pl.cluster) {
+    const int64_t total = M * (N / 8);
     const int threads = 256;
     splitk_reduce_kernel<<<unsigned((total + threads - 1) / threads), threads, 0, st>>>(
         static_cast<const int32_t*>(workspace), pl.splits, int(M), int(N), dx, dw, Y, ldy, acc_out);
@@ -1187,7 +1587,7 @@ int smoothrot_linear_static_scratch(const uint8_t* Xq, const float* dx, int64_t 
 size_t smoothrot_workspace_bytes(int64_t M, int64_t N, int64_t K) {
   if (M <= 0 || N <= 0 || K <= 0 || K % smoothrot::gemm::kWideRow != 0) return 0;
   const smoothrot::gemm::Plan pl = smoothrot::gemm::make_plan(M, N, K);
-  return pl.splits > 1 ? size_t(pl.splits) * size_t(M) * size_t(N) * sizeof(int32_t) : 0;
+  return (pl.splits > 1 && !pl.cluster) ? size_t(pl.splits) * size_t(M) * size_t(N) * sizeof(int32_t) : 0;
 }
 
 int smoothrot_linear(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq, const float* dw,

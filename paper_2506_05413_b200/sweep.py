@@ -1,0 +1,122 @@
+"""Token-count sweep over the linear shapes of one LLaMA-3.1-8B-shaped decoder block.
+
+    python -m paper_2506_05413_b200.sweep [--reps 30] [--json]
+
+For every shape (q/o 4096->4096, k/v 4096->1024, gate/up 4096->14336, down 14336->4096) and
+every M in {1, 4, 16, 128, 512, 2048, 8192} it times the two online calls of the layer,
+smoothrot_quant_act and smoothrot_linear, on seeded synthetic activations (random-init
+weights, quantized once by smoothrot_fuse_weights), and prints time, TOP/s and GB/s.
+
+Timing: each call is recorded into a CUDA graph per buffer set and replayed back to back
+between two CUDA events; the buffer sets rotate so that their total size exceeds twice the
+L2 capacity (weights included), which is what a decode step of a whole model sees.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import numpy as np
+
+from . import synth
+
+L2_BYTES = 126 * 1024 * 1024
+
+
+def _time_graphs(torch, graphs, reps):
+    n = len(graphs)
+    for i in range(max(3, n)):
+        graphs[i % n].replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(reps):
+        graphs[i % n].replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) * 1e-3 / reps      # seconds
+
+
+def run(reps: int = 30, shapes=None, tokens=None):
+    import torch
+    from . import binding as sr
+
+    sr.load()
+    dev = "cuda:0"
+    rows = []
+    for name, N, K in synth.BLOCK_SHAPES:
+        if shapes and name not in shapes:
+            continue
+        base = synth.config4(name, 8)                      # weights and diagonal do not depend on M
+        W = torch.from_numpy(base.W).to(dev)
+        d = torch.from_numpy(base.d).to(dev)
+        Xc = torch.from_numpy(base.X_calib).to(dev)
+        amax = torch.zeros(K, dtype=torch.float32, device=dev)
+        s, pre_w, pre_x = (torch.empty(K, dtype=torch.float32, device=dev) for _ in range(3))
+        sr.calibrate(Xc, amax, W=W, alpha=base.alpha, s_out=s, d=d, pre_w_out=pre_w, pre_x_out=pre_x)
+        for M in (tokens or synth.SWEEP_M):
+            case = synth.config4(name, M)
+            per_set = N * K // 2 + M * K * 2 + M * K // 2 + M * N * 2
+            n_sets = int(min(24, max(2, np.ceil(2.2 * L2_BYTES / per_set))))
+            sets = []
+            for _ in range(n_sets):
+                wq = torch.empty((N, K // 2), dtype=torch.uint8, device=dev)
+                dw = torch.empty(N, dtype=torch.float32, device=dev)
+                sr.fuse_weights(W, pre_w, case.clip_w, wq, dw)
+                X = torch.from_numpy(case.X).to(dev)
+                xq = torch.empty((M, K // 2), dtype=torch.uint8, device=dev)
+                dx = torch.empty(M, dtype=torch.float32, device=dev)
+                Y = torch.empty((M, N), dtype=torch.float16, device=dev)
+                need = sr.workspace_bytes(M, N, K)
+                ws = torch.empty(need, dtype=torch.uint8, device=dev) if need else None
+                sr.quant_act(X, pre_x, case.clip_a, xq, dx)
+                sr.linear(xq, dx, wq, dw, Y, ws)
+                sets.append((X, xq, dx, wq, dw, Y, ws))
+            torch.cuda.synchronize()
+            gq, gl = [], []
+            for X, xq, dx, wq, dw, Y, ws in sets:
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    sr.quant_act(X, pre_x, case.clip_a, xq, dx)
+                gq.append(g)
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    sr.linear(xq, dx, wq, dw, Y, ws)
+                gl.append(g)
+            tq = _time_graphs(torch, gq, reps)
+            tl = _time_graphs(torch, gl, reps)
+            assert sr.device_status() == 0
+            ops = 2.0 * M * N * K
+            rows.append({
+                "shape": name, "N": N, "K": K, "M": M,
+                "quant_act_us": tq * 1e6, "quant_act_GBs": (2.5 * M * K + 4 * M + 4 * K) / tq / 1e9,
+                "linear_us": tl * 1e6, "linear_TOPS": ops / tl / 1e12,
+                "linear_GBs": (0.5 * M * K + 0.5 * N * K + 2.0 * M * N + 4 * (M + N)) / tl / 1e9,
+                "weight_stream_GBs": 0.5 * N * K / tl / 1e9,
+                "buffer_sets": n_sets,
+            })
+            del sets, gq, gl
+            torch.cuda.empty_cache()
+    return rows
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--reps", type=int, default=30)
+    ap.add_argument("--json", action="store_true")
+    ap.add_argument("--shapes", nargs="*")
+    ap.add_argument("--tokens", nargs="*", type=int)
+    args = ap.parse_args()
+    rows = run(args.reps, args.shapes, args.tokens)
+    if args.json:
+        for r in rows:
+            print(json.dumps(r))
+        return
+    print(f"{'shape':8s} {'M':>5s} {'quant us':>9s} {'GB/s':>7s} {'linear us':>10s} {'TOP/s':>8s} {'W GB/s':>8s}")
+    for r in rows:
+        print(f"{r['shape']:8s} {r['M']:5d} {r['quant_act_us']:9.1f} {r['quant_act_GBs']:7.0f} "
+              f"{r['linear_us']:10.1f} {r['linear_TOPS']:8.1f} {r['weight_stream_GBs']:8.0f}")
+
+
+if __name__ == "__main__":
+    main()

@@ -165,6 +165,12 @@ GEMM_SHAPES = [
     (256, 256, 128),     # one two-CTA pair tile
     (600, 776, 512),     # two-CTA tiles, ragged in both directions
     (512, 1024, 14336),  # long K
+    (3, 1000, 1024),     # streaming kernel, 2 k-splits added up inside a cluster, ragged channels
+    (8, 520, 4096),      # 8 k-splits in a cluster
+    (40, 136, 2048),     # 64-token tile, 4 k-splits in a cluster
+    (128, 1024, 4096),   # 128-token tile, cluster
+    (4, 256, 16384),     # few channels, long K: k-splits through the workspace
+    (128, 256, 8192),
 ]
 
 
@@ -189,7 +195,8 @@ def test_gemm_extreme_codes(gu):
 
 
 @pytest.mark.parametrize("M,N,K", [(64, 256, 128), (3, 1024, 4096), (200, 264, 512), (130, 520, 4096),
-                                   (300, 520, 640), (1024, 768, 4096)])
+                                   (300, 520, 640), (1024, 768, 4096), (16, 1000, 2048), (128, 520, 1024),
+                                   (4, 256, 16384)])
 def test_linear_output_matches_oracle_on_gpu_codes(gu, M, N, K):
     rng = np.random.default_rng(M + N + K)
     xq = orc.pack_codes(synth.random_codes(M, M, K))

@@ -34,7 +34,8 @@ def test_static_scratch_entry_point_matches_linear_twice_in_a_row():
     build.build()
     dev = "cuda:0"
     t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
-    shapes = [(4, 1024, 4096), (16, 4096, 4096)]      # both split K (need scratch)
+    # few output channels and a long K: the shapes whose k-splits still go through scratch memory
+    shapes = [(4, 256, 16384), (16, 256, 32768)]
     for call, (M, N, K) in enumerate(shapes):
         need = sr.workspace_bytes(M, N, K)
         assert 0 < need <= sr.STATIC_SCRATCH_BYTES
@@ -58,7 +59,7 @@ def test_static_scratch_entry_point_refuses_oversized_shapes_and_needs_no_scratc
     from paper_2506_05413_b200 import build, binding as sr
     build.build()
     dev = "cuda:0"
-    M, N, K = 100, 14336, 4096                          # split-K partials beyond the built-in array
+    M, N, K = 128, 256, 37888                           # split-K partials beyond the built-in array
     assert sr.workspace_bytes(M, N, K) > sr.STATIC_SCRATCH_BYTES
     xq = torch.zeros((M, K // 2), dtype=torch.uint8, device=dev)
     wq = torch.zeros((N, K // 2), dtype=torch.uint8, device=dev)
