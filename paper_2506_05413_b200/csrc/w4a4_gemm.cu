@@ -956,8 +956,11 @@ struct Stream {
   static constexpr int kPackedStageBytes = kPackedA + kPackedBPad;
   static constexpr int kWideB = BN * kWideRow;
   static constexpr int kWideBPad = (kWideB + 1023) / 1024 * 1024;
-  static constexpr int kAWidenWarps = 4, kBWidenWarps = BN >= 128 ? 4 : (BN >= 64 ? 2 : 1);
-  static constexpr int kArrivals = kAWidenWarps + kBWidenWarps;
+  // with the 128-token tile two sets of widen warps take the k-blocks in turn
+  static constexpr int kSets = BN >= 128 ? 2 : 1;
+  static constexpr int kBPerSet = BN >= 128 ? 4 : (BN >= 64 ? 2 : 1);
+  static constexpr int kAWidenWarps = 4 * kSets, kBWidenWarps = kBPerSet * kSets;
+  static constexpr int kArrivals = 4 + kBPerSet;          // per k-block
   static constexpr int kThreads = 32 * (2 + kAWidenWarps + kBWidenWarps + kEpiWarps);
   static constexpr int kNumBarriers = 2 * kStages + 2 * kPackedStages + 1;
   static constexpr int kSmemBytes = 1024 + kStages * kWideBPad + kPackedStages * kPackedStageBytes +
@@ -1071,9 +1074,10 @@ w4a4_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
   } else if (warp < 2 + T::kAWidenWarps) {
     // ------------------------------------------------------------ A-widen warps: packed weight rows -> tensor memory
     const int q = warp & 3;
+    const int set = (warp - 2) >> 2;
     const int row = q * 32 + lane;
     const uint32_t sw = uint32_t((row >> 1) & 3);
-    for (int it = 0; it < kb_count; ++it) {
+    for (int it = set; it < kb_count; it += T::kSets) {
       const int ps = it % T::kPackedStages;
       const uint32_t pph = uint32_t(it / T::kPackedStages) & 1u;
       const int s = it % T::kStages;
@@ -1108,11 +1112,12 @@ w4a4_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     }
   } else if (warp < 2 + T::kAWidenWarps + T::kBWidenWarps) {
     // ------------------------------------------------------------ B-widen warps: packed token rows -> int8 tile
-    const int w = warp - 2 - T::kAWidenWarps;
+    const int w = (warp - 2 - T::kAWidenWarps) % T::kBPerSet;
+    const int set = (warp - 2 - T::kAWidenWarps) / T::kBPerSet;
     const int r = lane & 7;
     const int c = lane >> 3;
     constexpr int kGroups = BN / 8;
-    for (int it = 0; it < kb_count; ++it) {
+    for (int it = set; it < kb_count; it += T::kSets) {
       const int ps = it % T::kPackedStages;
       const uint32_t pph = uint32_t(it / T::kPackedStages) & 1u;
       const int s = it % T::kStages;
@@ -1122,7 +1127,7 @@ w4a4_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
       const uint32_t pk = packed_base + ps * T::kPackedStageBytes + T::kPackedA;
       const uint32_t wd = wide_base + s * T::kWideBPad;
 #pragma unroll
-      for (int g = w; g < kGroups; g += T::kBWidenWarps) {
+      for (int g = w; g < kGroups; g += T::kBPerSet) {
         const int row = g * 8 + r;
         const uint32_t src = pk + row * kPackedRow + ((c ^ ((row >> 1) & 3)) << 4);
         const uint32_t dst_row = wd + row * kWideRow;
@@ -1316,7 +1321,11 @@ static int sm_count() {
 static Plan make_plan(int64_t M, int64_t N, int64_t K) {
   Plan pl{};
   const int kblocks = int(K / kWideRow);
-  if (M > 128) {
+  // Up to 512 tokens the two-CTA kernel's 256 x 256 tiles can leave most SM pairs idle (few output
+  // channels); the streaming kernel with 128-token tiles and k-splits then fills the machine better.
+  const int64_t pair_tiles = ((M + 255) / 256) * ((N + 255) / 256);
+  const bool few_pair_tiles = M <= 512 && 16 * pair_tiles <= sm_count();
+  if (M > 128 && !few_pair_tiles) {
     pl.swapped = false;
     pl.pair = M >= 256 && N >= 256;
     pl.bn = (N >= 256) ? 256 : (N > 64 ? 128 : 64);
@@ -1325,7 +1334,7 @@ static Plan make_plan(int64_t M, int64_t N, int64_t K) {
   }
   pl.swapped = true;
   pl.bn = M <= 16 ? 16 : (M <= 32 ? 32 : (M <= 64 ? 64 : 128));
-  const int tiles = int((N + kBM - 1) / kBM);
+  const int tiles = int((N + kBM - 1) / kBM) * int((M + pl.bn - 1) / pl.bn);
   // two CTAs of the streaming kernel share an SM, except with the 128-token tile
   const int slots = (pl.bn <= 64 ? 2 : 1) * sm_count();
   int want = (slots + tiles - 1) / tiles;

@@ -171,6 +171,8 @@ GEMM_SHAPES = [
     (128, 1024, 4096),   # 128-token tile, cluster
     (4, 256, 16384),     # few channels, long K: k-splits through the workspace
     (128, 256, 8192),
+    (300, 1024, 2048),   # 3 token tiles of the streaming kernel, ragged
+    (512, 520, 1024),
 ]
 
 
