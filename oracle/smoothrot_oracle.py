@@ -19,6 +19,8 @@ What follows the paper, by passage:
 * Section "Experimental settings", paragraph "Quantization": 4 bits,
   per-token symmetric activations with clip ratio 0.9, per-output-channel
   symmetric round-to-nearest weights.
+* Fig. 2 (the feed-forward block): the down-projection input is the gated
+  product sigma(gate) (.) up; quant_act_glu takes that edge in one step.
 
 Floating point: transforms and scales are computed in float64 and rounded once
 to float32; the quantizer decisions (step, division, rounding) are taken in
@@ -282,6 +284,30 @@ def quant_act(X: np.ndarray, pre_x, K: int, clip_a: float = 0.9):
     Lambda^-1 already sits in the producing layer), rotated, quantized per
     token.  Returns (packed [M, K/2] u8, step [M] f32, rotated float32 [M, K])."""
     xr = rotate(X, pre_x, K).astype(np.float32)
+    codes, step = quantize_rows(xr, clip_a)
+    return pack_codes(codes), step, xr
+
+
+def silu(g: np.ndarray) -> np.ndarray:
+    """sigma(g) * g with the logistic function sigma, float64 (the GLU activation of Fig. 2:
+    the down-projection input is sigma(gate) (.) up, the two outputs of the fused gate/up layer)."""
+    g = np.asarray(g, dtype=np.float64)
+    with np.errstate(over="ignore"):
+        return g / (1.0 + np.exp(-g))
+
+
+def glu_product(gate: np.ndarray, up: np.ndarray) -> np.ndarray:
+    """The down-projection input of Fig. 2: SiLU(gate) * up, element by element, float64,
+    not rounded to fp16 (the fused kernel never stores it)."""
+    return silu(gate) * np.asarray(up, dtype=np.float64)
+
+
+def quant_act_glu(gate: np.ndarray, up: np.ndarray, pre_x, K: int, clip_a: float = 0.9):
+    """Online activation path fed by the gated linear unit: the edge
+    "x -> hadamard -> quantize" of Fig. 2 in one step.  Rows SiLU(gate) * up (float64), times
+    pre_x (or None: Lambda^-1 already sits in the up-projection), rotated, quantized per token.
+    Returns (packed [M, K/2] u8, step [M] f32, rotated float32 [M, K])."""
+    xr = rotate(glu_product(gate, up), pre_x, K).astype(np.float32)
     codes, step = quantize_rows(xr, clip_a)
     return pack_codes(codes), step, xr
 
