@@ -117,6 +117,21 @@ int smoothrot_quant_act(const void* X_f16, int64_t M, int64_t K, int64_t ldx,
                         uint8_t* Xq_out, float* dx_out, void* stream);
 
 /*
+ * The online activation path fed directly by the gated linear unit (Fig. 2: the edge
+ * "sigma(gate) (.) up -> hadamard -> quantize" in front of the down-projection; Methodology
+ * section: Lambda^-1 is absorbed into the up-projection because the gated product is
+ * channel-wise, so `pre` is normally NULL or the sign diagonal alone).  Same as
+ * smoothrot_quant_act on X[m][j] = SiLU(gate[m][j]) * up[m][j], SiLU(g) = g / (1 + exp(-g)),
+ * except that X is formed in fp32 inside the kernel and never rounded to fp16 or written to
+ * memory.  gate, up: [M x K] fp16 with leading dimensions ld_gate, ld_up (multiples of 8,
+ * 16-byte aligned rows).  K = 14336 runs the dedicated kernel; other supported K run the generic
+ * one-row-per-block kernel.
+ */
+int smoothrot_quant_act_glu(const void* gate_f16, const void* up_f16, int64_t M, int64_t K,
+                            int64_t ld_gate, int64_t ld_up, const float* pre, float clip_a,
+                            uint8_t* Xq_out, float* dx_out, void* stream);
+
+/*
  * The quantized layer (Eq. 2's product on the integer codes of Eq. 1, then
  * Eq. 1's dequantizer Q(x) = x_int * step applied to both factors):
  *     acc[m][n] = sum_k Xq[m][k] * Wq[n][k]                    (int32, exact)

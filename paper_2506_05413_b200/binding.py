@@ -24,6 +24,7 @@ SIGNATURES = {
     "smoothrot_calibrate": (_int, [_vp, _i64, _i64, _i64, _vp, _i64, _i64, _f32, _int, _vp, _vp, _vp, _vp, _vp, _vp]),
     "smoothrot_fuse_weights": (_int, [_vp, _i64, _i64, _i64, _vp, _f32, _vp, _vp, _vp]),
     "smoothrot_quant_act": (_int, [_vp, _i64, _i64, _i64, _vp, _f32, _vp, _vp, _vp]),
+    "smoothrot_quant_act_glu": (_int, [_vp, _vp, _i64, _i64, _i64, _i64, _vp, _f32, _vp, _vp, _vp]),
     "smoothrot_linear": (_int, [_vp, _vp, _i64, _vp, _vp, _i64, _i64, _vp, _i64, _vp, _sz, _vp]),
     "smoothrot_linear_static_scratch": (_int, [_vp, _vp, _i64, _vp, _vp, _i64, _i64, _vp, _i64, _vp]),
     "smoothrot_workspace_bytes": (_sz, [_i64, _i64, _i64]),
@@ -139,6 +140,19 @@ def fuse_weights(W, pre, clip_w, Wq_out, dw_out):
 def quant_act(X, pre, clip_a, Xq_out, dx_out):
     """smoothrot_quant_act: X [M, K] fp16 -> Xq_out [M, K/2] u8, dx_out [M] f32."""
     _quantize(load().smoothrot_quant_act, X, pre, clip_a, Xq_out, dx_out, ("X", "Xq_out", "dx_out"))
+
+
+def quant_act_glu(gate, up, pre, clip_a, Xq_out, dx_out):
+    """smoothrot_quant_act_glu: SiLU(gate) * up [M, K] (both fp16) -> Xq_out [M, K/2] u8, dx_out [M] f32."""
+    gp, R, K, ldg = _rows(gate, torch.float16, "gate")
+    up_p, Ru, Ku, ldu = _rows(up, torch.float16, "up")
+    if (Ru, Ku) != (R, K):
+        raise ValueError("gate and up must have the same shape")
+    if Xq_out.dtype != torch.uint8 or tuple(Xq_out.shape) != (R, K // 2) or not Xq_out.is_contiguous():
+        raise ValueError(f"Xq_out must be a contiguous uint8 [{R}, {K // 2}] tensor")
+    _check(load().smoothrot_quant_act_glu(gp, up_p, R, K, ldg, ldu, _vec(pre, K, "pre"), float(clip_a),
+                                          _ptr(Xq_out, torch.uint8, "Xq_out"), _vec(dx_out, R, "dx_out"),
+                                          _stream()))
 
 
 def workspace_bytes(M, N, K) -> int:

@@ -14,6 +14,8 @@
 //                           shared-memory transpose, codes assembled with warp
 //                           shuffles so that every global access is coalesced.
 //   paley512_kernel         K = 14336 = 28 x 512: see below.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace smoothrot {
@@ -97,14 +99,22 @@ __device__ __forceinline__ void unpack8_f16(const uint4& raw, float* f) {
   }
 }
 
+// SiLU(g) * u, the gated product of Fig. 2, in fp32 (fast exponential and division: relative
+// error below 1e-6, far inside the rotation tolerance).  Large |g| is safe: exp(-g) = inf gives
+// g / inf = -0, exp(-g) = 0 gives g.
+__device__ __forceinline__ float glu_product(float g, float u) {
+  return __fdividef(g, 1.0f + __expf(-g)) * u;
+}
+
 // ---------------------------------------------------------------------------
 // Generic kernel: one CTA per row.
 // ---------------------------------------------------------------------------
 constexpr int kGenericThreads = 256;
 
-template <bool kQuant>
+template <bool kQuant, bool kGlu>
 __global__ void __launch_bounds__(kGenericThreads)
-rotate_generic_kernel(const __half* __restrict__ X, int64_t ldx, int K, int base, int n, int logn,
+rotate_generic_kernel(const __half* __restrict__ X, int64_t ldx, const __half* __restrict__ U, int64_t ldu,
+                      int K, int base, int n, int logn,
                       const float* __restrict__ pre, float inv_sqrt_k, float clip,
                       uint8_t* __restrict__ q_out, float* __restrict__ step_out,
                       float* __restrict__ y_out) {
@@ -118,6 +128,13 @@ rotate_generic_kernel(const __half* __restrict__ X, int64_t ldx, int K, int base
     uint4 raw = *reinterpret_cast<const uint4*>(x + c * 8);
     float f[8];
     unpack8_f16(raw, f);
+    if (kGlu) {   // X holds the gate rows, U the up rows
+      const uint4 raw_u = *reinterpret_cast<const uint4*>(U + m * ldu + c * 8);
+      float u[8];
+      unpack8_f16(raw_u, u);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) f[i] = glu_product(f[i], u[i]);
+    }
     if (pre != nullptr) {
 #pragma unroll
       for (int i = 0; i < 8; ++i) f[i] *= pre[c * 8 + i];
@@ -616,18 +633,29 @@ struct Paley28Accumulate {
 };
 
 // One group of four inputs (rows a = 4G .. 4G+3 of the order-28 factor) of step 1.
-template <int G, bool kHasPre>
-__device__ __forceinline__ void paley28_group(f32x2* acc, uint32_t in_addr, const float* spre, int bp) {
+// With kGlu the value is SiLU(gate) * up, read from two input buffers kP512InBytes apart, and the
+// diagonal comes from global memory (shared memory is taken by the second input buffer).
+template <int G, bool kHasPre, bool kGlu>
+__device__ __forceinline__ void paley28_group(f32x2* acc, uint32_t in_addr, const float* pre_src, int bp) {
   f32x2 x[4];
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
     const int a = 4 * G + q;
     uint32_t raw;
     asm volatile("ld.shared.b32 %0, [%1];" : "=r"(raw) : "r"(in_addr + uint32_t(a * 1024 + bp * 4)) : "memory");
-    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&raw));
+    float2 f = __half22float2(*reinterpret_cast<const __half2*>(&raw));
+    if (kGlu) {
+      uint32_t raw_u;
+      asm volatile("ld.shared.b32 %0, [%1];"
+                   : "=r"(raw_u) : "r"(in_addr + uint32_t(kP512K * 2 + a * 1024 + bp * 4)) : "memory");
+      const float2 u = __half22float2(*reinterpret_cast<const __half2*>(&raw_u));
+      f.x = glu_product(f.x, u.x);
+      f.y = glu_product(f.y, u.y);
+    }
     x[q] = pack2(f.x, f.y);
     if (kHasPre) {
-      const float2 p = *reinterpret_cast<const float2*>(spre + a * 512 + bp * 2);
+      const float2 p = kGlu ? __ldg(reinterpret_cast<const float2*>(pre_src + a * 512 + bp * 2))
+                            : *reinterpret_cast<const float2*>(pre_src + a * 512 + bp * 2);
       x[q] = mul2(x[q], pack2(p.x, p.y));
     }
   }
@@ -654,29 +682,37 @@ __device__ __forceinline__ void group_barrier224(int group) {
   asm volatile("bar.sync %0, 224;" ::"r"(group + 1) : "memory");
 }
 
-template <bool kQuant, bool kHasPre, bool kLowClamp>
+// kGlu: the row is SiLU(gate) * up of two fp16 inputs (X = gate rows, U = up rows); the second
+// input buffer takes the place of the diagonal's copy in shared memory (same total).
+template <bool kQuant, bool kHasPre, bool kLowClamp, bool kGlu>
 __global__ void __launch_bounds__(kP512Threads, 1)
-paley512_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
+paley512_kernel(const __half* __restrict__ X, int64_t ldx, const __half* __restrict__ U, int64_t ldu, int64_t M,
                 const float* __restrict__ pre, float clip,
                 uint8_t* __restrict__ q_out, float* __restrict__ step_out,
                 float* __restrict__ y_out) {
   // shared memory: [pre: 14336 fp32][per group: input row fp16 | transformed row fp32][mbarriers][flags]
+  // with kGlu:     [per group: gate row fp16 | up row fp16 | transformed row fp32][mbarriers][flags]
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __shared__ float red[kP512Groups][8];   // one slot per warp of a group (7 used)
+  constexpr int kPreBytes = kGlu ? 0 : kP512PreBytes;
+  constexpr int kInBytes = kGlu ? 2 * kP512InBytes : kP512InBytes;
+  constexpr int kGroupBytes = kInBytes + kP512RowBytes;
+  static_assert(kPreBytes + kP512Groups * kGroupBytes == kP512PreBytes + kP512Groups * kP512GroupBytes,
+                "both layouts fill the same shared memory");
   const int group = threadIdx.x >= kP512GroupThreads ? 1 : 0;
   const int t = threadIdx.x - group * kP512GroupThreads;
   const int lane = threadIdx.x & 31;
-  float* spre = reinterpret_cast<float*>(smem_raw);
-  uint8_t* gbase = smem_raw + kP512PreBytes + group * kP512GroupBytes;
+  const float* spre = kGlu ? pre : reinterpret_cast<const float*>(smem_raw);   // where step 1 reads the diagonal
+  uint8_t* gbase = smem_raw + kPreBytes + group * kGroupBytes;
   const uint32_t inbuf = smem_addr(gbase);
-  float* row = reinterpret_cast<float*>(gbase + kP512InBytes);
+  float* row = reinterpret_cast<float*>(gbase + kInBytes);
   const uint32_t bar = smem_addr(smem_raw + kP512PreBytes + kP512Groups * kP512GroupBytes + group * 8);
   volatile int* lost = reinterpret_cast<volatile int*>(smem_raw + kP512PreBytes + kP512Groups * kP512GroupBytes +
                                                        kP512Groups * 8) + group;
 
-  if (kHasPre) {
+  if (kHasPre && !kGlu) {
     for (int i = threadIdx.x; i < kP512K / 4; i += kP512Threads)
-      reinterpret_cast<float4*>(spre)[i] = __ldg(reinterpret_cast<const float4*>(pre) + i);
+      reinterpret_cast<float4*>(smem_raw)[i] = __ldg(reinterpret_cast<const float4*>(pre) + i);
   }
   if (t == 0) {
     *lost = 0;
@@ -685,9 +721,24 @@ paley512_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
   }
   __syncthreads();
 
+  // one row (or the gate and up rows) into the group's input buffer, completion on `bar`
+  auto fetch_row = [&](int64_t r) {
+    if (kGlu) {
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                   ::"r"(bar), "r"(uint32_t(2 * kP512InBytes)) : "memory");
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                   ::"r"(inbuf), "l"(X + r * ldx), "r"(uint32_t(kP512InBytes)), "r"(bar) : "memory");
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                   ::"r"(inbuf + uint32_t(kP512InBytes)), "l"(U + r * ldu), "r"(uint32_t(kP512InBytes)), "r"(bar)
+                   : "memory");
+    } else {
+      start_row_copy(inbuf, X + r * ldx, kP512InBytes, bar);
+    }
+  };
+
   const int64_t stride = int64_t(gridDim.x) * kP512Groups;
   int64_t m = int64_t(blockIdx.x) + int64_t(gridDim.x) * group;
-  if (t == 0 && m < M) start_row_copy(inbuf, X + m * ldx, kP512InBytes, bar);
+  if (t == 0 && m < M) fetch_row(m);
   uint32_t parity = 0;
 
   // step 2 ownership: row a of the order-28 factor, lane group j
@@ -701,13 +752,13 @@ paley512_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
     //      first warp of the group takes a second pair
     for (int bp = t; bp < 256; bp += kP512GroupThreads) {
       f32x2 acc[28];
-      paley28_group<0, kHasPre>(acc, inbuf, spre, bp);
-      paley28_group<1, kHasPre>(acc, inbuf, spre, bp);
-      paley28_group<2, kHasPre>(acc, inbuf, spre, bp);
-      paley28_group<3, kHasPre>(acc, inbuf, spre, bp);
-      paley28_group<4, kHasPre>(acc, inbuf, spre, bp);
-      paley28_group<5, kHasPre>(acc, inbuf, spre, bp);
-      paley28_group<6, kHasPre>(acc, inbuf, spre, bp);
+      paley28_group<0, kHasPre, kGlu>(acc, inbuf, spre, bp);
+      paley28_group<1, kHasPre, kGlu>(acc, inbuf, spre, bp);
+      paley28_group<2, kHasPre, kGlu>(acc, inbuf, spre, bp);
+      paley28_group<3, kHasPre, kGlu>(acc, inbuf, spre, bp);
+      paley28_group<4, kHasPre, kGlu>(acc, inbuf, spre, bp);
+      paley28_group<5, kHasPre, kGlu>(acc, inbuf, spre, bp);
+      paley28_group<6, kHasPre, kGlu>(acc, inbuf, spre, bp);
       // fp32 row [28][512], its 16-byte units permuted by p512_unit
       const int phys = p512_unit(bp >> 1);
 #pragma unroll
@@ -719,7 +770,7 @@ paley512_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
     }
     group_barrier224(group);   // input consumed, transformed row complete
     if (*lost != 0) break;
-    if (t == 0 && m + stride < M) start_row_copy(inbuf, X + (m + stride) * ldx, kP512InBytes, bar);
+    if (t == 0 && m + stride < M) fetch_row(m + stride);
 
     // ---- step 2: Walsh-512 along b ------------------------------------------------------------
     f32x2 v[32];
@@ -866,14 +917,23 @@ static int check_rows(const void* X, int64_t rows, int64_t K, int64_t ld, int* b
   return SMOOTHROT_OK;
 }
 
+// U != nullptr: X holds gate rows, U up rows, and the transformed row is SiLU(gate) * up.
 template <bool kQuant>
-static int launch_rotate(const void* X, int64_t rows, int64_t K, int64_t ld, const float* pre, float clip,
-                         uint8_t* q_out, float* step_out, float* y_out, cudaStream_t stream) {
+static int launch_rotate(const void* X, int64_t rows, int64_t K, int64_t ld, const void* U, int64_t ldu,
+                         const float* pre, float clip, uint8_t* q_out, float* step_out, float* y_out,
+                         cudaStream_t stream) {
   int base = 0, n = 0, logn = 0;
   int rc = check_rows(X, rows, K, ld, &base, &n, &logn);
   if (rc != SMOOTHROT_OK || rows == 0) return rc;
+  const bool glu = U != nullptr;
+  if (glu) {
+    int b2 = 0, n2 = 0, l2 = 0;
+    rc = check_rows(U, rows, K, ldu, &b2, &n2, &l2);
+    if (rc != SMOOTHROT_OK) return rc;
+  }
   const __half* x = static_cast<const __half*>(X);
-  if (K == 4096) {
+  const __half* u = static_cast<const __half*>(U);
+  if (K == 4096 && !glu) {
     // codes below -8 can only come up when the row maximum sits at 8.5 steps or more
     const bool low = kQuant && (7.0f / clip >= 8.49f);
     auto kern = pre ? (low ? walsh4096_kernel<kQuant, true, true> : walsh4096_kernel<kQuant, true, false>)
@@ -888,33 +948,37 @@ static int launch_rotate(const void* X, int64_t rows, int64_t K, int64_t ld, con
   }
   if (K == kP512K) {
     const bool low = kQuant && (7.0f / clip >= 8.49f);
-    auto kern = pre ? (low ? paley512_kernel<kQuant, true, true> : paley512_kernel<kQuant, true, false>)
-                    : (low ? paley512_kernel<kQuant, false, true> : paley512_kernel<kQuant, false, false>);
+    auto pick = [&](auto glu_tag) {
+      constexpr bool kG = decltype(glu_tag)::value;
+      return pre ? (low ? paley512_kernel<kQuant, true, true, kG> : paley512_kernel<kQuant, true, false, kG>)
+                 : (low ? paley512_kernel<kQuant, false, true, kG> : paley512_kernel<kQuant, false, false, kG>);
+    };
+    auto kern = glu ? pick(std::true_type{}) : pick(std::false_type{});
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kP512SmemBytes) != cudaSuccess)
       return SMOOTHROT_CUDA_ERROR;
     const int sms = device_sm_count();
     const unsigned grid = unsigned(rows < sms ? rows : sms);
-    kern<<<grid, kP512Threads, kP512SmemBytes, stream>>>(x, ld, rows, pre, clip, q_out, step_out, y_out);
+    kern<<<grid, kP512Threads, kP512SmemBytes, stream>>>(x, ld, u, ldu, rows, pre, clip, q_out, step_out, y_out);
     count_launch();
     return launch_status();
   }
   const size_t smem = size_t(K) * sizeof(float);
-  auto kern = rotate_generic_kernel<kQuant>;
+  auto kern = glu ? rotate_generic_kernel<kQuant, true> : rotate_generic_kernel<kQuant, false>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
     return SMOOTHROT_CUDA_ERROR;
   const float inv_sqrt_k = float(1.0 / sqrt(double(K)));
-  kern<<<unsigned(rows), kGenericThreads, smem, stream>>>(x, ld, int(K), base, n, logn, pre, inv_sqrt_k, clip,
+  kern<<<unsigned(rows), kGenericThreads, smem, stream>>>(x, ld, u, ldu, int(K), base, n, logn, pre, inv_sqrt_k, clip,
                                                            q_out, step_out, y_out);
   count_launch();
   return launch_status();
 }
 
-static int quantize_entry(const void* X, int64_t rows, int64_t K, int64_t ld, const float* pre, float clip,
-                          uint8_t* q_out, float* step_out, void* stream) {
+static int quantize_entry(const void* X, int64_t rows, int64_t K, int64_t ld, const void* U, int64_t ldu,
+                          const float* pre, float clip, uint8_t* q_out, float* step_out, void* stream) {
   if (!(clip > 0.0f) || clip > 1.0f) return SMOOTHROT_INVALID_ARG;
   if (rows > 0 && (q_out == nullptr || step_out == nullptr)) return SMOOTHROT_INVALID_ARG;
   if (rows > 0 && (!aligned16(q_out) || (pre != nullptr && !aligned16(pre)))) return SMOOTHROT_BAD_ALIGNMENT;
-  return launch_rotate<true>(X, rows, K, ld, pre, clip, q_out, step_out, nullptr,
+  return launch_rotate<true>(X, rows, K, ld, U, ldu, pre, clip, q_out, step_out, nullptr,
                              static_cast<cudaStream_t>(stream));
 }
 
@@ -924,19 +988,26 @@ extern "C" {
 
 int smoothrot_fuse_weights(const void* W_f16, int64_t N, int64_t K, int64_t ldw, const float* pre,
                            float clip_w, uint8_t* Wq_out, float* dw_out, void* stream) {
-  return smoothrot::quantize_entry(W_f16, N, K, ldw, pre, clip_w, Wq_out, dw_out, stream);
+  return smoothrot::quantize_entry(W_f16, N, K, ldw, nullptr, 0, pre, clip_w, Wq_out, dw_out, stream);
 }
 
 int smoothrot_quant_act(const void* X_f16, int64_t M, int64_t K, int64_t ldx, const float* pre,
                         float clip_a, uint8_t* Xq_out, float* dx_out, void* stream) {
-  return smoothrot::quantize_entry(X_f16, M, K, ldx, pre, clip_a, Xq_out, dx_out, stream);
+  return smoothrot::quantize_entry(X_f16, M, K, ldx, nullptr, 0, pre, clip_a, Xq_out, dx_out, stream);
+}
+
+int smoothrot_quant_act_glu(const void* gate_f16, const void* up_f16, int64_t M, int64_t K, int64_t ld_gate,
+                            int64_t ld_up, const float* pre, float clip_a, uint8_t* Xq_out, float* dx_out,
+                            void* stream) {
+  if (M > 0 && up_f16 == nullptr) return SMOOTHROT_INVALID_ARG;
+  return smoothrot::quantize_entry(gate_f16, M, K, ld_gate, up_f16, ld_up, pre, clip_a, Xq_out, dx_out, stream);
 }
 
 int smoothrot_debug_hadamard(const void* X_f16, int64_t M, int64_t K, int64_t ldx, const float* pre,
                              float* Y_f32, void* stream) {
   if (M > 0 && Y_f32 == nullptr) return SMOOTHROT_INVALID_ARG;
   if (M > 0 && pre != nullptr && !smoothrot::aligned16(pre)) return SMOOTHROT_BAD_ALIGNMENT;
-  return smoothrot::launch_rotate<false>(X_f16, M, K, ldx, pre, 1.0f, nullptr, nullptr, Y_f32,
+  return smoothrot::launch_rotate<false>(X_f16, M, K, ldx, nullptr, 0, pre, 1.0f, nullptr, nullptr, Y_f32,
                                          static_cast<cudaStream_t>(stream));
 }
 

@@ -251,3 +251,53 @@ def test_config0_whole_layer(gu):
 def test_reduced_configs_whole_layer(gu, maker, M, N):
     case = maker(M=M, N=N)
     _check_layer(gu, case, _layer_on_gpu(gu, case))
+
+
+# ------------------------------------------------ gated-linear-unit input path
+@pytest.mark.parametrize("K,M", [(128, 9), (512, 21), (4096, 5), (28 * 16, 10), (14336, 1), (14336, 37)])
+@pytest.mark.parametrize("use_pre", [False, True])
+def test_glu_quantized_codes_match_oracle(gu, K, M, use_pre):
+    import torch
+    from paper_2506_05413_b200 import binding as sr
+    rng = np.random.default_rng(K + M)
+    gate = (rng.standard_normal((M, K)) * 2.0).astype(np.float16)
+    up = rng.standard_normal((M, K)).astype(np.float16)
+    gate[0, :7] = [0.0, -65504.0, 65504.0, 30.0, -30.0, 11.0, -11.0]     # the ends of the SiLU
+    up[min(1, M - 1), 3] = 2000.0                                        # a massive outlier
+    pre = _pre(K + 3, K) if use_pre else None
+    q = torch.empty((M, K // 2), dtype=torch.uint8, device=gu.DEV)
+    step = torch.empty(M, dtype=torch.float32, device=gu.DEV)
+    sr.quant_act_glu(gu.dev(gate), gu.dev(up), gu.dev(pre) if use_pre else None, 0.9, q, step)
+    torch.cuda.synchronize()
+    assert sr.device_status() == 0
+    q_ref, step_ref, _ = orc.quant_act_glu(gate, up, pre, K, 0.9)
+    # the kernel evaluates the SiLU in fp32 with fast exp / divide: 1e-6 on the largest entry of a row
+    assert np.abs(step.cpu().numpy() / step_ref - 1).max() <= 2e-6
+    frac, worst = gu.code_mismatch(q.cpu().numpy(), q_ref)
+    assert worst <= 1 and frac <= max(2 * TOL_CODES, 1.5 / q.numel() / 2)
+
+
+def test_glu_path_equals_plain_path_when_the_product_is_exact_in_fp16(gu):
+    """gate = 30 makes SiLU(gate) = 30 to fp32 precision; with up a multiple of 1/32 the product is an
+    fp16 number, so the fused call and quant_act on that fp16 matrix must agree."""
+    import torch
+    from paper_2506_05413_b200 import binding as sr
+    rng = np.random.default_rng(5)
+    for K in (512, 14336):
+        M = 6
+        up = (rng.integers(-64, 65, size=(M, K)) / 32.0).astype(np.float16)
+        gate = np.full((M, K), 30.0, np.float16)
+        X = (30.0 * up.astype(np.float64)).astype(np.float16)
+        outs = []
+        for call in ("glu", "plain"):
+            q = torch.empty((M, K // 2), dtype=torch.uint8, device=gu.DEV)
+            step = torch.empty(M, dtype=torch.float32, device=gu.DEV)
+            if call == "glu":
+                sr.quant_act_glu(gu.dev(gate), gu.dev(up), None, 0.9, q, step)
+            else:
+                sr.quant_act(gu.dev(X), None, 0.9, q, step)
+            torch.cuda.synchronize()
+            outs.append((q.cpu().numpy(), step.cpu().numpy()))
+        assert np.abs(outs[0][1] / outs[1][1] - 1).max() <= 2e-6
+        frac, worst = gu.code_mismatch(outs[0][0], outs[1][0])
+        assert worst <= 1 and frac <= 1e-3
