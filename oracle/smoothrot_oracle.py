@@ -279,6 +279,47 @@ def fuse_weights(W: np.ndarray, pre_w, K: int, clip_w: float = 1.0):
     return pack_codes(codes), step, wr
 
 
+def clip_ratios(count: int = 51, lowest: float = 0.5) -> np.ndarray:
+    """The grid of the weight clip search: `count` ratios from 1.0 down to `lowest`, equally
+    spaced, as float32.  The paper only says that the ratio is found by a linear search over the
+    squared error; the grid is this repository's reading."""
+    i = np.arange(count, dtype=np.float64)
+    return (1.0 - i * (1.0 - lowest) / (count - 1)).astype(np.float32)
+
+
+def clip_search_rows(v: np.ndarray, ratios: np.ndarray):
+    """Per row of the float32 matrix v: quantize with every clip ratio of the grid (Eq. 1,
+    symmetric, step = float32(ratio * max|v|) / 7, all decisions in float32 as in quantize_rows),
+    measure the squared error  sum_k (v_k - code_k * step)^2  in float64, and keep the first ratio
+    that attains the minimum (the largest such ratio).
+    Returns (codes int8 [R, C], step float32 [R], best index [R], errors float64 [R, len(ratios)])."""
+    v = np.asarray(v, dtype=np.float32)
+    R = v.shape[0]
+    errs = np.empty((R, len(ratios)), dtype=np.float64)
+    all_codes, all_steps = [], []
+    for i, ratio in enumerate(ratios):
+        codes, step = quantize_rows(v, np.float32(ratio))
+        deq = codes.astype(np.float64) * step.astype(np.float64)[:, None]
+        errs[:, i] = ((v.astype(np.float64) - deq) ** 2).sum(axis=1)
+        all_codes.append(codes)
+        all_steps.append(step)
+    best = np.argmin(errs, axis=1)          # first minimum
+    rows = np.arange(R)
+    codes = np.stack(all_codes)[best, rows]
+    step = np.stack(all_steps)[best, rows]
+    return codes, step, best, errs
+
+
+def fuse_weights_search(W: np.ndarray, pre_w, K: int, ratios: np.ndarray):
+    """Offline weight path with the clip-ratio search of the paper's weight quantizer
+    (Experimental settings, "Quantization": clipping ratios found by a linear search over the
+    squared error): rotate as in fuse_weights, then clip_search_rows per output channel.
+    Returns (packed [N, K/2] u8, step [N] f32, best index [N], errors [N, len(ratios)], rotated f32)."""
+    wr = rotate(W, pre_w, K).astype(np.float32)
+    codes, step, best, errs = clip_search_rows(wr, ratios)
+    return pack_codes(codes), step, best, errs, wr
+
+
 def quant_act(X: np.ndarray, pre_x, K: int, clip_a: float = 0.9):
     """Online activation path: rows times pre_x (= d / s, or None when
     Lambda^-1 already sits in the producing layer), rotated, quantized per
