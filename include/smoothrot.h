@@ -101,6 +101,25 @@ int smoothrot_fuse_weights(const void* W_f16, int64_t N, int64_t K, int64_t ldw,
                            uint8_t* Wq_out, float* dw_out, void* stream);
 
 /*
+ * Offline weight path with the clip-ratio search of the paper's weight quantizer (Experimental
+ * settings, "Quantization": per-channel symmetric weights whose "clipping ratios [are] determined
+ * through a linear search over the squared error").  As smoothrot_fuse_weights, but for every row
+ * the ratio is chosen from the grid
+ *     ratio_i = fp32(1 - i * (1 - lowest_ratio) / (ratio_count - 1)),   i = 0 .. ratio_count - 1
+ * (the paper gives no grid; 1.00 .. 0.50 in 51 steps is what the tests and the oracle use) as the
+ * first i that minimises  sum_k (w^_k - code_k * step_i)^2,  step_i = fp32(ratio_i * max|w^|) / 7,
+ * with the codes of Eq. 1's symmetric quantizer at that step; the error is summed in fp64.
+ * best_out [N] int32 (may be NULL) receives the chosen i.  `workspace` holds the rotated fp32
+ * rows: smoothrot_fuse_weights_search_workspace_bytes(N, K) bytes for one pass, or any multiple
+ * of 4 K bytes (at least one row) to work in slices.  0 < lowest_ratio <= 1, 1 <= ratio_count <= 1024.
+ */
+size_t smoothrot_fuse_weights_search_workspace_bytes(int64_t N, int64_t K);
+int smoothrot_fuse_weights_search(const void* W_f16, int64_t N, int64_t K, int64_t ldw,
+                                  const float* pre, float lowest_ratio, int ratio_count,
+                                  uint8_t* Wq_out, float* dw_out, int32_t* best_out,
+                                  void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Online activation path (Fig. 2, "hadamard" then "quantize" before the
  * down-projection; Experimental settings, "Quantization": per-token symmetric
  * 4-bit activations with a constant clip ratio, 0.9 in the paper).  For every

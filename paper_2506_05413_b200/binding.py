@@ -23,6 +23,8 @@ SIGNATURES = {
     "smoothrot_status_string": (ctypes.c_char_p, [_int]),
     "smoothrot_calibrate": (_int, [_vp, _i64, _i64, _i64, _vp, _i64, _i64, _f32, _int, _vp, _vp, _vp, _vp, _vp, _vp]),
     "smoothrot_fuse_weights": (_int, [_vp, _i64, _i64, _i64, _vp, _f32, _vp, _vp, _vp]),
+    "smoothrot_fuse_weights_search_workspace_bytes": (_sz, [_i64, _i64]),
+    "smoothrot_fuse_weights_search": (_int, [_vp, _i64, _i64, _i64, _vp, _f32, _int, _vp, _vp, _vp, _vp, _sz, _vp]),
     "smoothrot_quant_act": (_int, [_vp, _i64, _i64, _i64, _vp, _f32, _vp, _vp, _vp]),
     "smoothrot_quant_act_glu": (_int, [_vp, _vp, _i64, _i64, _i64, _i64, _vp, _f32, _vp, _vp, _vp]),
     "smoothrot_linear": (_int, [_vp, _vp, _i64, _vp, _vp, _i64, _i64, _vp, _i64, _vp, _sz, _vp]),
@@ -135,6 +137,25 @@ def _quantize(fn, X, pre, clip, q_out, step_out, names):
 def fuse_weights(W, pre, clip_w, Wq_out, dw_out):
     """smoothrot_fuse_weights: W [N, K] fp16 -> Wq_out [N, K/2] u8, dw_out [N] f32."""
     _quantize(load().smoothrot_fuse_weights, W, pre, clip_w, Wq_out, dw_out, ("W", "Wq_out", "dw_out"))
+
+
+def fuse_weights_search(W, pre, lowest_ratio, ratio_count, Wq_out, dw_out, best_out=None, workspace=None):
+    """smoothrot_fuse_weights_search: as fuse_weights, with the per-row clip ratio chosen from the grid
+    1 .. lowest_ratio (ratio_count values) by least squared error.  best_out [N] int32 is optional;
+    workspace (uint8) must hold at least one rotated fp32 row, ideally all N."""
+    wp, N, K, ld = _rows(W, torch.float16, "W")
+    if Wq_out.dtype != torch.uint8 or tuple(Wq_out.shape) != (N, K // 2) or not Wq_out.is_contiguous():
+        raise ValueError(f"Wq_out must be a contiguous uint8 [{N}, {K // 2}] tensor")
+    wsp = _ptr(workspace, None, "workspace")
+    wsb = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    _check(load().smoothrot_fuse_weights_search(
+        wp, N, K, ld, _vec(pre, K, "pre"), float(lowest_ratio), int(ratio_count),
+        _ptr(Wq_out, torch.uint8, "Wq_out"), _vec(dw_out, N, "dw_out"),
+        _vec(best_out, N, "best_out", torch.int32), wsp, wsb, _stream()))
+
+
+def fuse_weights_search_workspace_bytes(N, K) -> int:
+    return int(load().smoothrot_fuse_weights_search_workspace_bytes(int(N), int(K)))
 
 
 def quant_act(X, pre, clip_a, Xq_out, dx_out):

@@ -301,3 +301,42 @@ def test_glu_path_equals_plain_path_when_the_product_is_exact_in_fp16(gu):
         assert np.abs(outs[0][1] / outs[1][1] - 1).max() <= 2e-6
         frac, worst = gu.code_mismatch(outs[0][0], outs[1][0])
         assert worst <= 1 and frac <= 1e-3
+
+
+# ------------------------------------------------ weight clip-ratio search
+@pytest.mark.parametrize("K,N,slices", [(128, 40, 1), (4096, 33, 1), (4096, 9, 4), (14336, 10, 1), (28 * 16, 12, 3)])
+def test_weight_clip_search_matches_oracle(gu, K, N, slices):
+    import torch
+    from paper_2506_05413_b200 import binding as sr
+    rng = np.random.default_rng(K + N)
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float16)
+    W[1, 5] = 0.9                                   # a row with a far outlier: clipping pays
+    W[2, :] = 0                                     # an all-zero row
+    W[3, :] = 0; W[3, 7] = 0.25                     # a single entry: flat after rotation, ratio 1 is exact
+    pre = _pre(K + 11, K)
+    ratios = orc.clip_ratios(51, 0.5)
+    q = torch.empty((N, K // 2), dtype=torch.uint8, device=gu.DEV)
+    step = torch.empty(N, dtype=torch.float32, device=gu.DEV)
+    best = torch.full((N,), -1, dtype=torch.int32, device=gu.DEV)
+    full = sr.fuse_weights_search_workspace_bytes(N, K)
+    assert full == N * K * 4
+    ws_bytes = full if slices == 1 else (N // slices + 1) * K * 4 + 64     # not a multiple of a row on purpose
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=gu.DEV)
+    sr.fuse_weights_search(gu.dev(W), gu.dev(pre), 0.5, 51, q, step, best, ws)
+    torch.cuda.synchronize()
+    q, step, best = q.cpu().numpy(), step.cpu().numpy(), best.cpu().numpy()
+    packed_ref, step_ref, best_ref, errs, wr = orc.fuse_weights_search(W, pre, K, ratios)
+    assert best.min() >= 0 and best.max() < 51
+    rows = np.arange(N)
+    # the chosen ratio minimises the oracle's error curve (up to the fp32 noise of the rotation)
+    assert np.all(errs[rows, best] <= errs.min(axis=1) * (1 + 1e-4) + 1e-30)
+    assert (best != best_ref).mean() <= 0.1
+    assert best[2] == 0 and step[2] == np.float32(1.0) and best[3] == 0
+    # staged: the oracle's quantizer at the ratio the GPU chose
+    for r in rows:
+        codes_r, step_r = orc.quantize_rows(wr[r:r + 1], ratios[best[r]])
+        assert abs(step[r] / step_r[0] - 1) <= TOL_SCALE
+        a = orc.unpack_codes(q[r:r + 1]).astype(int)
+        diff = np.abs(a - codes_r.astype(int))
+        assert diff.max() <= 1 and (diff != 0).mean() <= max(TOL_CODES, 1.5 / K)
+    assert best[1] > 0          # the outlier row took a smaller ratio
