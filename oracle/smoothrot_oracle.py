@@ -19,6 +19,8 @@ What follows the paper, by passage:
 * Section "Experimental settings", paragraph "Quantization": 4 bits,
   per-token symmetric activations with clip ratio 0.9, per-output-channel
   symmetric round-to-nearest weights.
+* Eq. 1, asymmetric form, and "Quantization": KV caches with asymmetric
+  quantization, group size 128 and clip ratio 0.95 (kv_quantize).
 * Fig. 2 (the feed-forward block): the down-projection input is the gated
   product sigma(gate) (.) up; quant_act_glu takes that edge in one step.
 
@@ -263,6 +265,59 @@ def unpack_codes(packed: np.ndarray) -> np.ndarray:
 def dequantize_rows(codes: np.ndarray, step: np.ndarray) -> np.ndarray:
     """Q(x) = x_int * step  (Eq. 1's dequantizer, zero point 0), float64."""
     return codes.astype(np.float64) * np.asarray(step, dtype=np.float64)[:, None]
+
+
+# ---------------------------------------------------------------------------
+# KV-cache quantizer (Eq. 1, asymmetric form; Experimental settings: asymmetric,
+# group size 128, clip ratio 0.95)
+# ---------------------------------------------------------------------------
+KV_GROUP = 128
+
+
+def kv_quantize(X: np.ndarray, clip: float = 0.95, group: int = KV_GROUP):
+    """Asymmetric 4-bit quantization of each group of `group` consecutive values of a row.
+    Eq. 1's asymmetric form with the clip ratio shrinking both ends of the range:
+        hi = float32(clip * max),  lo = float32(clip * min)
+        step = (hi - lo) / 15            (1.0 if hi == lo: a constant group; a reading, the
+                                          paper does not treat the degenerate case)
+        zero = -round_half_even(lo / step)
+        code = clamp(round_half_even(x / step) + zero, 0, 15)
+    All decisions in float32.  Returns (codes uint8 [R, C] in 0..15, step f32 [R, C/group],
+    zero f32 [R, C/group], integer valued)."""
+    X = np.asarray(X)
+    R, C = X.shape
+    assert C % group == 0
+    x = X.astype(np.float32).reshape(R, C // group, group)
+    hi = (np.float32(clip) * x.max(axis=2)).astype(np.float32)
+    lo = (np.float32(clip) * x.min(axis=2)).astype(np.float32)
+    step = ((hi - lo).astype(np.float32) / np.float32(15.0)).astype(np.float32)
+    step = np.where(hi == lo, np.float32(1.0), step).astype(np.float32)
+    zero = (-np.rint((lo / step).astype(np.float32))).astype(np.float32)
+    q = np.rint((x / step[:, :, None]).astype(np.float32)) + zero[:, :, None]
+    codes = np.clip(q, 0, 15).astype(np.uint8).reshape(R, C)
+    return codes, step, zero
+
+
+def kv_dequantize(codes: np.ndarray, step: np.ndarray, zero: np.ndarray, group: int = KV_GROUP) -> np.ndarray:
+    """Q(x) = (x_int - zero) * step  (Eq. 1's dequantizer), float64, [R, C]."""
+    R, C = codes.shape
+    c = codes.astype(np.float64).reshape(R, C // group, group)
+    y = (c - zero.astype(np.float64)[:, :, None]) * step.astype(np.float64)[:, :, None]
+    return y.reshape(R, C)
+
+
+def pack_nibbles(codes: np.ndarray) -> np.ndarray:
+    """[R, C] uint8 codes in 0..15 -> [R, C/2] uint8, value 2i in bits 0-3, value 2i+1 in bits 4-7."""
+    c = np.asarray(codes, dtype=np.uint8)
+    return (c[..., 0::2] | (c[..., 1::2] << 4)).astype(np.uint8)
+
+
+def unpack_nibbles(packed: np.ndarray) -> np.ndarray:
+    p = np.asarray(packed, dtype=np.uint8)
+    out = np.empty(p.shape[:-1] + (p.shape[-1] * 2,), dtype=np.uint8)
+    out[..., 0::2] = p & 0xF
+    out[..., 1::2] = p >> 4
+    return out
 
 
 # ---------------------------------------------------------------------------
