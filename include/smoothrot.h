@@ -203,6 +203,24 @@ int smoothrot_linear_static_scratch(const uint8_t* Xq, const float* dx, int64_t 
                                     const uint8_t* Wq, const float* dw, int64_t N, int64_t K,
                                     void* Y_f16, int64_t ldy, void* stream);
 
+/*
+ * KV-cache quantizer (Eq. 1, asymmetric form; Experimental settings, "Quantization": KV caches
+ * are quantized asymmetrically with a group size of 128 and a clip ratio of 0.95).  For every
+ * group of 128 consecutive values of a row of X [rows x C] fp16 (C a multiple of 128):
+ *     hi = fp32(clip * max), lo = fp32(clip * min)        (the ratio shrinks both ends)
+ *     step = (hi - lo) / 15                               (1.0 for a constant group)
+ *     zero = -round_half_even(lo / step)
+ *     code = clamp(round_half_even(x / step) + zero, 0, 15)
+ * all in fp32.  q_out [rows x C/2] bytes holds the unsigned codes, value 2i in bits 0-3 and value
+ * 2i+1 in bits 4-7; step_out, zero_out [rows x C/128] fp32 (zero is integer valued and may lie
+ * outside 0..15 when a group does not straddle zero).  0 < clip <= 1.
+ * smoothrot_kv_dequant is Eq. 1's dequantizer  Y = fp16((code - zero) * step),  Y [rows x ldy].
+ */
+int smoothrot_kv_quant(const void* X_f16, int64_t rows, int64_t C, int64_t ldx, float clip,
+                       uint8_t* q_out, float* step_out, float* zero_out, void* stream);
+int smoothrot_kv_dequant(const uint8_t* q, const float* step, const float* zero, int64_t rows,
+                         int64_t C, void* Y_f16, int64_t ldy, void* stream);
+
 /* Host. Scratch bytes smoothrot_linear / smoothrot_debug_gemm_i32 need for
  * this shape (0 for shapes that need none). */
 size_t smoothrot_workspace_bytes(int64_t M, int64_t N, int64_t K);

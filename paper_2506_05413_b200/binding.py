@@ -27,6 +27,8 @@ SIGNATURES = {
     "smoothrot_fuse_weights_search": (_int, [_vp, _i64, _i64, _i64, _vp, _f32, _int, _vp, _vp, _vp, _vp, _sz, _vp]),
     "smoothrot_quant_act": (_int, [_vp, _i64, _i64, _i64, _vp, _f32, _vp, _vp, _vp]),
     "smoothrot_quant_act_glu": (_int, [_vp, _vp, _i64, _i64, _i64, _i64, _vp, _f32, _vp, _vp, _vp]),
+    "smoothrot_kv_quant": (_int, [_vp, _i64, _i64, _i64, _f32, _vp, _vp, _vp, _vp]),
+    "smoothrot_kv_dequant": (_int, [_vp, _vp, _vp, _i64, _i64, _vp, _i64, _vp]),
     "smoothrot_linear": (_int, [_vp, _vp, _i64, _vp, _vp, _i64, _i64, _vp, _i64, _vp, _sz, _vp]),
     "smoothrot_linear_static_scratch": (_int, [_vp, _vp, _i64, _vp, _vp, _i64, _i64, _vp, _i64, _vp]),
     "smoothrot_workspace_bytes": (_sz, [_i64, _i64, _i64]),
@@ -174,6 +176,31 @@ def quant_act_glu(gate, up, pre, clip_a, Xq_out, dx_out):
     _check(load().smoothrot_quant_act_glu(gp, up_p, R, K, ldg, ldu, _vec(pre, K, "pre"), float(clip_a),
                                           _ptr(Xq_out, torch.uint8, "Xq_out"), _vec(dx_out, R, "dx_out"),
                                           _stream()))
+
+
+KV_GROUP = 128
+
+
+def kv_quant(X, clip, q_out, step_out, zero_out):
+    """smoothrot_kv_quant: X [R, C] fp16 -> q_out [R, C/2] u8, step_out / zero_out [R, C/128] f32."""
+    xp, R, C, ld = _rows(X, torch.float16, "X")
+    if q_out.dtype != torch.uint8 or tuple(q_out.shape) != (R, C // 2) or not q_out.is_contiguous():
+        raise ValueError(f"q_out must be a contiguous uint8 [{R}, {C // 2}] tensor")
+    for t, name in ((step_out, "step_out"), (zero_out, "zero_out")):
+        if t.dtype != torch.float32 or tuple(t.shape) != (R, C // KV_GROUP) or not t.is_contiguous():
+            raise ValueError(f"{name} must be a contiguous float32 [{R}, {C // KV_GROUP}] tensor")
+    _check(load().smoothrot_kv_quant(xp, R, C, ld, float(clip), _ptr(q_out, torch.uint8, "q_out"),
+                                     _ptr(step_out, torch.float32, "step_out"),
+                                     _ptr(zero_out, torch.float32, "zero_out"), _stream()))
+
+
+def kv_dequant(q, step, zero, Y):
+    """smoothrot_kv_dequant: Y [R, C] fp16 = (code - zero) * step."""
+    yp, R, C, ld = _rows(Y, torch.float16, "Y")
+    if q.dtype != torch.uint8 or tuple(q.shape) != (R, C // 2) or not q.is_contiguous():
+        raise ValueError(f"q must be a contiguous uint8 [{R}, {C // 2}] tensor")
+    _check(load().smoothrot_kv_dequant(_ptr(q, torch.uint8, "q"), _ptr(step, torch.float32, "step"),
+                                       _ptr(zero, torch.float32, "zero"), R, C, yp, ld, _stream()))
 
 
 def workspace_bytes(M, N, K) -> int:

@@ -340,3 +340,50 @@ def test_weight_clip_search_matches_oracle(gu, K, N, slices):
         diff = np.abs(a - codes_r.astype(int))
         assert diff.max() <= 1 and (diff != 0).mean() <= max(TOL_CODES, 1.5 / K)
     assert best[1] > 0          # the outlier row took a smaller ratio
+
+
+# ------------------------------------------------ KV-cache quantizer
+@pytest.mark.parametrize("R,C", [(1, 128), (7, 1024), (300, 512), (4099, 256)])
+@pytest.mark.parametrize("clip", [0.95, 1.0, 0.6])
+def test_kv_quantizer_matches_oracle_and_round_trips(gu, R, C, clip):
+    """Steps and zero points come from the same fp32 operations on both sides and must be identical.
+    The codes are decided in fp32 on both sides too, but the kernel multiplies by the rounded
+    reciprocal of the step where the oracle divides: at most 1e-4 of them may differ, by one.
+    The dequantizer is checked on the GPU's own codes, within one fp16 rounding."""
+    import torch
+    from paper_2506_05413_b200 import binding as sr
+    rng = np.random.default_rng(R + C)
+    X = rng.standard_normal((R, C)).astype(np.float16)
+    X[0, :128] = 2.5                                  # a constant group
+    if R > 2:
+        X[1, :] = 0                                   # all zero
+        X[2, 5] = 300.0                               # an outlier: the clip ratio saturates it
+        X[2, 128 * (C // 128 - 1):] = np.abs(X[2, 128 * (C // 128 - 1):]) + 1   # a group that does not straddle zero
+    pad = torch.zeros((R, C + 8), dtype=torch.float16, device=gu.DEV)      # a strided input
+    pad[:, :C] = gu.dev(X)
+    q = torch.empty((R, C // 2), dtype=torch.uint8, device=gu.DEV)
+    step = torch.empty((R, C // 128), dtype=torch.float32, device=gu.DEV)
+    zero = torch.empty((R, C // 128), dtype=torch.float32, device=gu.DEV)
+    sr.kv_quant(pad[:, :C], clip, q, step, zero)
+    Y = torch.empty((R, C), dtype=torch.float16, device=gu.DEV)
+    sr.kv_dequant(q, step, zero, Y)
+    torch.cuda.synchronize()
+    codes_ref, step_ref, zero_ref = orc.kv_quantize(X, clip)
+    assert np.array_equal(step.cpu().numpy(), step_ref)
+    assert np.array_equal(zero.cpu().numpy(), zero_ref)
+    codes_gpu = orc.unpack_nibbles(q.cpu().numpy())
+    diff = np.abs(codes_gpu.astype(int) - codes_ref.astype(int))
+    assert diff.max() <= 1 and (diff != 0).mean() <= TOL_CODES
+    want = orc.kv_dequantize(codes_gpu, step_ref, zero_ref)
+    got = Y.cpu().numpy().astype(np.float64)
+    assert np.allclose(got, want, rtol=1e-3, atol=1e-7)
+
+
+def test_kv_quantizer_rejects_bad_arguments(gu):
+    import torch
+    from paper_2506_05413_b200 import binding as sr
+    X = torch.zeros((2, 192), dtype=torch.float16, device=gu.DEV)           # not a multiple of 128
+    q = torch.empty((2, 96), dtype=torch.uint8, device=gu.DEV)
+    s = torch.empty((2, 1), dtype=torch.float32, device=gu.DEV)
+    with pytest.raises(sr.SmoothRotError):
+        sr.kv_quant(X, 0.95, q, s, s.clone())
