@@ -230,13 +230,13 @@ rotate_generic_kernel(const __half* __restrict__ X, int64_t ldx, const __half* _
 }
 
 // ---------------------------------------------------------------------------
-// K = 4096.  Persistent kernel: one CTA per SM, kW4096Groups row groups of 64
-// threads (two warps) each; a group walks over rows  m, m + stride, ...
+// K = 4096.  Persistent kernel: one CTA per SM, kW4096Groups (12) row groups of
+// 64 threads (two warps) each; a group walks over rows  m, m + stride, ...
 //
 // The next row of a group is fetched by a bulk asynchronous copy
-// (cp.async.bulk, completion on an mbarrier) into the group's own 8 KB input
-// buffer while the current row is being transformed, so that the 8 groups of
-// an SM keep up to 64 KB of loads in flight and HBM never waits for arithmetic.
+// (cp.async.bulk, completion on an mbarrier) into the group's transpose tile as
+// soon as the tile has been read back (midway through the current row), so that
+// loads stay in flight while the second half of the row's arithmetic runs.
 //
 // Index bits of a row position j (12 bits):  i = j[0:3), t = j[3:9), g = j[9:12).
 //   phase 1  thread t reads the eight 16-byte chunks (g, t): values (g, i);
@@ -248,13 +248,13 @@ rotate_generic_kernel(const __half* __restrict__ X, int64_t ldx, const __half* _
 //   codes travel between the lanes of a row group so that each lane ends up
 //   with whole 32-bit words of packed output.
 // ---------------------------------------------------------------------------
-constexpr int kW4096Groups = 8;
+constexpr int kW4096Groups = 10;
 constexpr int kW4096Threads = kW4096Groups * 64;
 constexpr int kW4096Pitch = 68;  // floats per t-row in shared memory (64 + 4 pad)
 constexpr int kW4096PreBytes = 4096 * 4;
 constexpr int kW4096TileBytes = 64 * kW4096Pitch * 4;
 constexpr int kW4096InBytes = 4096 * 2;
-constexpr int kW4096GroupBytes = kW4096TileBytes + kW4096InBytes;
+constexpr int kW4096GroupBytes = kW4096TileBytes;   // the next row lands in the tile's first 8 KB
 constexpr int kW4096SmemBytes = kW4096PreBytes + kW4096Groups * kW4096GroupBytes + kW4096Groups * 8 + kW4096Groups * 4;
 constexpr unsigned long long kLoadWaitLimitNs = 2000000000ull;  // 2 s
 
@@ -357,6 +357,37 @@ __device__ __forceinline__ void butterflies_pairs(f32x2* v) {
   }
 }
 
+// The stage inside each pair with instructions that stay where they are written: they consume
+// every value just loaded from shared memory, so that the loads have completed before the code
+// that follows (a barrier, then a bulk copy into the same memory) can run.
+template <int NP>
+__device__ __forceinline__ void butterflies_first_stage_in_place(f32x2* v) {
+#pragma unroll
+  for (int k = 0; k < NP; ++k) {
+    float a, b, s, d;
+    unpack2(v[k], a, b);
+    asm volatile("add.f32 %0, %1, %2;" : "=f"(s) : "f"(a), "f"(b));
+    asm volatile("sub.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    v[k] = pack2(s, d);
+  }
+}
+
+// The remaining stages (between pairs) of butterflies_pairs.
+template <int NP>
+__device__ __forceinline__ void butterflies_between_pairs(f32x2* v) {
+#pragma unroll
+  for (int h = 1; h < NP; h <<= 1) {
+#pragma unroll
+    for (int k = 0; k < NP; ++k) {
+      if ((k & h) == 0) {
+        const f32x2 a = v[k], b = v[k + h];
+        v[k] = add2(a, b);
+        v[k + h] = sub2(a, b);
+      }
+    }
+  }
+}
+
 // kLowClamp: the general two-sided clamp, needed when the row maximum can reach 8.5 steps or more
 // (clip ratios <= 7/8.5); otherwise only the code +8 can occur out of range and is fixed on the bytes.
 template <bool kQuant, bool kHasPre, bool kLowClamp>
@@ -365,7 +396,8 @@ walsh4096_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
                  const float* __restrict__ pre, float clip,
                  uint8_t* __restrict__ q_out, float* __restrict__ step_out,
                  float* __restrict__ y_out) {
-  // shared memory: [pre: 4096 fp32][per group: transpose tile | input row][per group: mbarrier][per group: flag]
+  // shared memory: [pre: 4096 fp32][per group: transpose tile, also the landing place of the next row]
+  //                [per group: mbarrier][per group: flag]
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __shared__ float red[kW4096Groups][2];
   const int group = threadIdx.x >> 6;
@@ -374,7 +406,7 @@ walsh4096_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
   float* spre = reinterpret_cast<float*>(smem_raw);
   uint8_t* gbase = smem_raw + kW4096PreBytes + group * kW4096GroupBytes;
   float* tile = reinterpret_cast<float*>(gbase);
-  const uint32_t inbuf = smem_addr(gbase + kW4096TileBytes);
+  const uint32_t inbuf = smem_addr(gbase);   // the input row shares the tile
   const uint32_t bar = smem_addr(smem_raw + kW4096PreBytes + kW4096Groups * kW4096GroupBytes + group * 8);
   volatile int* lost = reinterpret_cast<volatile int*>(smem_raw + kW4096PreBytes + kW4096Groups * kW4096GroupBytes +
                                                          kW4096Groups * 8) + group;
@@ -412,9 +444,8 @@ walsh4096_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
       asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
                    : "=r"(raw[g].x), "=r"(raw[g].y), "=r"(raw[g].z), "=r"(raw[g].w)
                    : "r"(inbuf + uint32_t(g * 1024 + t * 16)) : "memory");
-    group_barrier(group);   // the whole row is in registers: the buffer can take the next row
+    group_barrier(group);   // the whole row is in registers: the tile can take the transposed values
     if (*lost != 0) break;
-    if (t == 0 && m + stride < M) start_row_copy(inbuf, X + (m + stride) * ldx, kW4096InBytes, bar);
 #pragma unroll
     for (int g = 0; g < 8; ++g) {
       const __half2* h = reinterpret_cast<const __half2*>(&raw[g]);
@@ -453,7 +484,10 @@ walsh4096_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
   // thread gi = t now owns position (g, i) = (t >> 3, t & 7) for all 64 values of the t-bits
 #pragma unroll
   for (int u = 0; u < 32; ++u) v[u] = pack2(tile[(2 * u) * kW4096Pitch + t], tile[(2 * u + 1) * kW4096Pitch + t]);
-  butterflies_pairs<32>(v);
+  butterflies_first_stage_in_place<32>(v);   // every loaded value has been consumed
+  group_barrier(group);                       // the tile is free: fetch the next row into it
+  if (t == 0 && m + stride < M) start_row_copy(inbuf, X + (m + stride) * ldx, kW4096InBytes, bar);
+  butterflies_between_pairs<32>(v);
 
   const int gi_g = t >> 3, gi_i = t & 7;
   if (!kQuant) {
