@@ -238,6 +238,16 @@ def gpu_step(sr, case, ds):
         fn()
 
 
+def max_over_ranks(torch, dist, value, dev):
+    """The slowest rank's figure (a time): what a multi-GPU number is quoted on.  `dist` is
+    torch.distributed (initialised) or None for a single process."""
+    if dist is None:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def capture(torch, fns):
     """Records the given calls (made through the binding, on the capturing stream) into one CUDA graph."""
     g = torch.cuda.CUDAGraph()
@@ -320,11 +330,7 @@ def run_gpu(args, case, desc):
     barrier()
     launches = launches_per_step * args.steps
     clocks = sampler.stop() if rank == 0 else None
-    total_ms = start.elapsed_time(stop)
-    if dist is not None:
-        tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
+    total_ms = max_over_ranks(torch, dist, start.elapsed_time(stop), dev)
     ms_per_step = total_ms / args.steps
     linear_live_ms = float(np.mean([ev[i][0].elapsed_time(ev[i][1]) for i in range(args.steps)]))
     assert sr.device_status() == 0, "a device-side wait timed out"
@@ -370,11 +376,7 @@ def run_gpu(args, case, desc):
     for _ in range(e2e_steps):
         e2e_step()
     barrier()
-    e2e_sec = (time.perf_counter() - t0) / e2e_steps
-    if dist is not None:
-        tt = torch.tensor([e2e_sec], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_sec = float(tt.item())
+    e2e_sec = max_over_ranks(torch, dist, (time.perf_counter() - t0) / e2e_steps, dev)
 
     if rank != 0:
         if dist is not None:
