@@ -23,10 +23,13 @@
 // The kernels are persistent (one CTA per SM, tiles handed out round-robin).
 // Shapes with M >= 256 and N >= 256 run the two-CTA kernel further down, which
 // keeps the token operand in tensor memory instead of shared memory.
-// For M < 128 tokens the roles of the operands are swapped (output channels on
+// For M <= 128 tokens the roles of the operands are swapped (output channels on
 // the 128-row MMA axis, tokens on the N axis) and K is split across CTAs;
-// the int32 partial sums go to the caller's workspace and a second kernel
-// adds them and dequantizes.
+// the int32 partial sums are added inside a thread-block cluster, or go to the
+// caller's workspace where a second kernel adds them and dequantizes.
+// For M <= 16 tokens none of this machinery pays: a small kernel streams the
+// weights with plain loads and forms the products with the warp-level integer
+// MMA (see the decode kernel near the end).
 //
 // Every wait on an mbarrier is bounded in wall time; a wait that runs out
 // sets a device status word, raises a CTA-wide abort flag and the kernel
@@ -1295,9 +1298,212 @@ splitk_reduce_kernel(const int32_t* __restrict__ part, int splits, int M, int N,
 }
 
 // ---------------------------------------------------------------------------
+// Decode kernel for M <= 16 tokens.
+//
+// With a handful of tokens the layer is one pass over the packed weights and nothing else,
+// and the tensor-memory kernels spend more time on their set-up (cluster launch, tensor-memory
+// allocation, barrier chains, a reduction over k-splits) than on the stream.  This kernel has
+// no set-up at all: a CTA of 8 warps owns 16 * RG weight rows, its warps take the rows'
+// 64-byte chunks in turn (a split of K inside the CTA), and every lane loads 16 bytes of two
+// weight rows and 16 bytes of one token's codes straight from global memory.  The products
+// are formed by the warp-level integer MMA (16 rows x 8 tokens x 32 codes per instruction),
+// used here as a dot-product engine for a kernel that is bound by HBM: its operands are the
+// same 16 * code int8 words as above (low nibbles and high nibbles of a packed word go to
+// different k slots of the instruction, for weights and tokens alike, and a dot product does
+// not care about the order of its terms).  Sums are int32 (256 * acc), added over the warps in
+// shared memory in a fixed order: exact, and identical from run to run.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void mma_s8_16x8x32(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Volatile so that every load of a batch is issued before the first MMA that follows it in the source.
+__device__ __forceinline__ uint4 load_stream_16(const uint8_t* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+__device__ __forceinline__ uint4 load_keep_16(const uint8_t* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ uint32_t even_codes_x16(uint32_t w) { return (w << 4) & 0xF0F0F0F0u; }
+__device__ __forceinline__ uint32_t odd_codes_x16(uint32_t w) { return w & 0xF0F0F0F0u; }
+__device__ __forceinline__ uint32_t word_of(const uint4& v, int i) { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
+
+// NT: token tiles of 8 (M <= 8 * NT); RG: row groups of 16 per CTA; U: chunks per batch and warp (two
+// batches are in flight); WARPS: warps per CTA, which split K between them.
+template <int NT, int RG, int U>
+struct DecodeBatch {
+  uint4 w[U][RG][2];
+  uint4 x[U][NT];
+};
+
+template <int NT, int RG, int U, int WARPS>
+__device__ __forceinline__ void decode_load(DecodeBatch<NT, RG, U>& b, const uint8_t* const (&wrow)[RG][2],
+                                            const uint8_t* const (&xrow)[NT], const bool (&xvalid)[NT], int c0,
+                                            int chunks) {
+  const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    const int cc = c0 + u * WARPS;
+    const bool on = cc < chunks;
+#pragma unroll
+    for (int rg = 0; rg < RG; ++rg)
+#pragma unroll
+      for (int h = 0; h < 2; ++h) b.w[u][rg][h] = on ? load_stream_16(wrow[rg][h] + cc * 64) : zero;
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) b.x[u][nt] = (on && xvalid[nt]) ? load_keep_16(xrow[nt] + cc * 64) : zero;
+  }
+}
+
+template <int NT, int RG, int U>
+__device__ __forceinline__ void decode_accumulate(const DecodeBatch<NT, RG, U>& b, int (&c)[RG][NT][4]) {
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      uint32_t b0[NT], b1[NT];
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        const uint32_t xw = word_of(b.x[u][nt], i);
+        b0[nt] = even_codes_x16(xw);
+        b1[nt] = odd_codes_x16(xw);
+      }
+#pragma unroll
+      for (int rg = 0; rg < RG; ++rg) {
+        const uint32_t wa = word_of(b.w[u][rg][0], i), wb = word_of(b.w[u][rg][1], i);
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+          mma_s8_16x8x32(c[rg][nt], even_codes_x16(wa), even_codes_x16(wb), odd_codes_x16(wa), odd_codes_x16(wb),
+                         b0[nt], b1[nt]);
+      }
+    }
+  }
+}
+
+template <int NT, int RG, int U, int WARPS, bool PIPE>
+__global__ void __launch_bounds__(WARPS * 32)
+w4a4_decode_kernel(const uint8_t* __restrict__ Xq, const uint8_t* __restrict__ Wq, int M, int N, int K,
+                   const float* __restrict__ dx, const float* __restrict__ dw, __half* __restrict__ Y, int64_t ldy,
+                   int32_t* __restrict__ acc_out) {
+  constexpr int kOutputs = RG * NT * 128;          // outputs of the CTA, tokens past M included
+  constexpr int kPerThread = (kOutputs + WARPS * 32 - 1) / (WARPS * 32);
+  __shared__ int red[WARPS][kOutputs];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int g = lane >> 2, t = lane & 3;
+  const int row_base = blockIdx.x * (16 * RG);
+  const int chunks = K / 128;                    // 64-byte chunks of a packed row
+  const int64_t row_bytes = K / 2;
+
+  // a row past the end repeats the last one, a token past the end contributes zeros
+  const uint8_t* wrow[RG][2];
+#pragma unroll
+  for (int rg = 0; rg < RG; ++rg)
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+      wrow[rg][h] = Wq + int64_t(min(row_base + rg * 16 + h * 8 + g, N - 1)) * row_bytes + t * 16;
+  const uint8_t* xrow[NT];
+  bool xvalid[NT];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    xvalid[nt] = nt * 8 + g < M;
+    xrow[nt] = Xq + int64_t(min(nt * 8 + g, M - 1)) * row_bytes + t * 16;
+  }
+
+  DecodeBatch<NT, RG, U> cur;
+  decode_load<NT, RG, U, WARPS>(cur, wrow, xrow, xvalid, warp, chunks);
+
+  // the scales of this thread's outputs arrive while the weights stream
+  float scale[kPerThread];
+#pragma unroll
+  for (int j = 0; j < kPerThread; ++j) {
+    const int o = threadIdx.x + j * WARPS * 32;
+    const int tile = o >> 7, i = o & 127;
+    const int m = (tile % NT) * 8 + (i >> 4);
+    const int n = row_base + (tile / NT) * 16 + (i & 15);
+    scale[j] = (Y != nullptr && o < kOutputs && m < M && n < N) ? __ldg(dx + m) * __ldg(dw + n) : 0.0f;
+  }
+
+  int c[RG][NT][4];
+#pragma unroll
+  for (int rg = 0; rg < RG; ++rg)
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) c[rg][nt][i] = 0;
+
+  if constexpr (PIPE) {                  // long rows: the next batch is on its way during the MMAs
+    DecodeBatch<NT, RG, U> nxt;
+    for (int c0 = warp; c0 < chunks; c0 += WARPS * U) {
+      const int c1 = c0 + WARPS * U;
+      if (c1 < chunks) decode_load<NT, RG, U, WARPS>(nxt, wrow, xrow, xvalid, c1, chunks);
+      decode_accumulate<NT, RG, U>(cur, c);
+      cur = nxt;
+    }
+  } else {                               // short rows: one batch (or few) per warp, more CTAs per SM instead
+    for (int c0 = warp; c0 < chunks; c0 += WARPS * U) {
+      if (c0 != warp) decode_load<NT, RG, U, WARPS>(cur, wrow, xrow, xvalid, c0, chunks);
+      decode_accumulate<NT, RG, U>(cur, c);
+    }
+  }
+
+  // lane (g, t) holds rows g and g + 8, tokens 2t and 2t + 1 of every 16 x 8 tile; tiles are
+  // laid out token-major in shared memory so that the final stores run along the channels
+#pragma unroll
+  for (int rg = 0; rg < RG; ++rg)
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      int* tile = &red[warp][(rg * NT + nt) * 128];
+      tile[(2 * t) * 16 + g] = c[rg][nt][0];
+      tile[(2 * t + 1) * 16 + g] = c[rg][nt][1];
+      tile[(2 * t) * 16 + g + 8] = c[rg][nt][2];
+      tile[(2 * t + 1) * 16 + g + 8] = c[rg][nt][3];
+    }
+  __syncthreads();
+#pragma unroll
+  for (int j = 0; j < kPerThread; ++j) {
+    const int o = threadIdx.x + j * WARPS * 32;
+    if (o < kOutputs) {
+      int sum = 0;
+#pragma unroll
+      for (int w = 0; w < WARPS; ++w) sum += red[w][o];
+      sum >>= 8;                                   // the sums are 256 * acc, exactly
+      const int tile = o >> 7, i = o & 127;
+      const int m = (tile % NT) * 8 + (i >> 4);
+      const int n = row_base + (tile / NT) * 16 + (i & 15);
+      if (m < M && n < N) {
+        if (Y != nullptr)
+          Y[int64_t(m) * ldy + n] = __float2half_rn(float(sum) * scale[j]);
+        else
+          acc_out[int64_t(m) * N + n] = sum;
+      }
+    }
+  }
+}
+
+template <int NT, int RG, int U, int WARPS, bool PIPE>
+static int launch_decode(const uint8_t* Xq, const uint8_t* Wq, int M, int N, int K, const float* dx, const float* dw,
+                         __half* Y, int64_t ldy, int32_t* acc_out, cudaStream_t st) {
+  const int grid = (N + 16 * RG - 1) / (16 * RG);
+  w4a4_decode_kernel<NT, RG, U, WARPS, PIPE><<<grid, WARPS * 32, 0, st>>>(Xq, Wq, M, N, K, dx, dw, Y, ldy, acc_out);
+  count_launch();
+  return launch_status();
+}
+
+// ---------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------
 struct Plan {
+  bool gemv;      // M <= 16: the decode kernel
   bool swapped;
   bool pair;      // two-CTA kernel, 256 x 256 pair tiles
   bool cluster;   // the k-splits of a tile form a cluster and add up in shared memory (no workspace)
@@ -1321,6 +1527,11 @@ static int sm_count() {
 static Plan make_plan(int64_t M, int64_t N, int64_t K) {
   Plan pl{};
   const int kblocks = int(K / kWideRow);
+  if (M <= 16) {                   // the decode kernel: no tiles, no k-splits, no workspace
+    pl.gemv = true;
+    pl.splits = 1;
+    return pl;
+  }
   // Up to 512 tokens the two-CTA kernel's 256 x 256 tiles can leave most SM pairs idle (few output
   // channels); the streaming kernel with 128-token tiles and k-splits then fills the machine better.
   const int64_t pair_tiles = ((M + 255) / 256) * ((N + 255) / 256);
@@ -1333,7 +1544,7 @@ static Plan make_plan(int64_t M, int64_t N, int64_t K) {
     return pl;
   }
   pl.swapped = true;
-  pl.bn = M <= 16 ? 16 : (M <= 32 ? 32 : (M <= 64 ? 64 : 128));
+  pl.bn = M <= 32 ? 32 : (M <= 64 ? 64 : 128);
   const int tiles = int((N + kBM - 1) / kBM) * int((M + pl.bn - 1) / pl.bn);
   // two CTAs of the streaming kernel share an SM, except with the 128-token tile
   const int slots = (pl.bn <= 64 ? 2 : 1) * sm_count();
@@ -1466,6 +1677,17 @@ static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq,
   if (need > 0 && (workspace == nullptr || workspace_bytes < need)) return SMOOTHROT_WORKSPACE_TOO_SMALL;
   if (need > 0 && !aligned16(workspace)) return SMOOTHROT_BAD_ALIGNMENT;
 
+  if (pl.gemv) {
+    // Short rows fit one batch of loads per warp, and many small CTAs per SM keep the memory system
+    // busy; long rows (K > 4096) want the double-buffered loop, and with two token tiles the codes of
+    // the tokens are worth sharing between two row groups.
+    int32_t* out32 = Y ? nullptr : acc_out;
+    const int m = int(M), n = int(N), k = int(K);
+#define SR_DECODE(NT, RG, U, W, P) launch_decode<NT, RG, U, W, P>(Xq, Wq, m, n, k, dx, dw, Y, ldy, out32, st)
+    if (M <= 8) return K > 4096 ? SR_DECODE(1, 1, 4, 8, true) : SR_DECODE(1, 1, 4, 8, false);
+    return K > 4096 ? SR_DECODE(2, 2, 2, 16, true) : SR_DECODE(2, 1, 4, 8, false);
+#undef SR_DECODE
+  }
   Params p{};
   p.swapped = pl.swapped ? 1 : 0;
   const uint8_t* a_ptr = pl.swapped ? Wq : Xq;
@@ -1514,8 +1736,7 @@ static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq,
     switch (pl.bn) {
       case 128: rc = launch_stream<128>(ma, mb, p, st); break;
       case 64: rc = launch_stream<64>(ma, mb, p, st); break;
-      case 32: rc = launch_stream<32>(ma, mb, p, st); break;
-      default: rc = launch_stream<16>(ma, mb, p, st); break;
+      default: rc = launch_stream<32>(ma, mb, p, st); break;
     }
   } else
   switch (pl.bn) {

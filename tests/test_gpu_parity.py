@@ -152,9 +152,23 @@ def test_calibration_matches_oracle(gu, K, T, N, batches):
 # --------------------------------------------------------------------- GEMM
 GEMM_SHAPES = [
     (64, 256, 128),      # config 0
-    (1, 1024, 4096),     # decode, split K
+    # M <= 16: the decode kernel (plain loads, warp-level integer MMA, K split between the warps of a CTA)
+    (1, 1024, 4096),
     (4, 4096, 4096),
-    (16, 136, 512),
+    (2, 1000, 1024),     # ragged channels (N % 16 == 8)
+    (3, 4104, 3072),
+    (4, 264, 14336),     # long rows: the double-buffered loop
+    (1, 8, 1024),
+    (3, 1000, 1152),     # fewer 64-byte chunks than a batch holds
+    (8, 1024, 4096),
+    (6, 4096, 4096),
+    (7, 72, 128),        # one chunk: seven of the eight warps have nothing to add
+    (16, 136, 512),      # two token tiles
+    (9, 264, 14336),     # two token tiles, long rows, 16 warps
+    (16, 1000, 8192),
+    (13, 520, 4224),     # long rows with a partial last batch
+    (8, 256, 16384),
+    # the streaming kernel
     (17, 64, 256),       # 32-wide token tile
     (33, 72, 384),       # 64-wide token tile
     (100, 264, 256),     # 128-wide token tile, swapped
@@ -165,11 +179,11 @@ GEMM_SHAPES = [
     (256, 256, 128),     # one two-CTA pair tile
     (600, 776, 512),     # two-CTA tiles, ragged in both directions
     (512, 1024, 14336),  # long K
-    (3, 1000, 1024),     # streaming kernel, 2 k-splits added up inside a cluster, ragged channels
-    (8, 520, 4096),      # 8 k-splits in a cluster
+    (17, 1000, 1024),    # streaming kernel, 2 k-splits added up inside a cluster, ragged channels
+    (20, 520, 4096),     # 8 k-splits in a cluster
     (40, 136, 2048),     # 64-token tile, 4 k-splits in a cluster
     (128, 1024, 4096),   # 128-token tile, cluster
-    (4, 256, 16384),     # few channels, long K: k-splits through the workspace
+    (24, 256, 16384),    # few channels, long K: k-splits through the workspace
     (128, 256, 8192),
     (300, 1024, 2048),   # 3 token tiles of the streaming kernel, ragged
     (512, 520, 1024),
@@ -198,7 +212,8 @@ def test_gemm_extreme_codes(gu):
 
 @pytest.mark.parametrize("M,N,K", [(64, 256, 128), (3, 1024, 4096), (200, 264, 512), (130, 520, 4096),
                                    (300, 520, 640), (1024, 768, 4096), (16, 1000, 2048), (128, 520, 1024),
-                                   (4, 256, 16384)])
+                                   (24, 256, 16384), (4, 1000, 14336), (1, 4096, 4096), (6, 1024, 4096), (16, 520, 14336),
+                                   (12, 4104, 2048), (32, 1024, 4096)])
 def test_linear_output_matches_oracle_on_gpu_codes(gu, M, N, K):
     rng = np.random.default_rng(M + N + K)
     xq = orc.pack_codes(synth.random_codes(M, M, K))
