@@ -161,15 +161,6 @@ __device__ __forceinline__ void tmem_load32(uint32_t taddr, uint32_t* r) {
       : "r"(taddr)
       : "memory");
 }
-__device__ __forceinline__ void tmem_load16(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
-}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of
@@ -434,20 +425,12 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       tcgen05_fence_after();
       const int a = ta * kBM + e * 32 + lane;
       const uint32_t taddr = tmem_base + (uint32_t(e * 32) << 16) + uint32_t(ab * BN);
-      if constexpr (BN >= 32) {
 #pragma unroll 1
-        for (int c0 = 0; c0 < BN; c0 += 32) {
-          uint32_t regs[32];
-          tmem_load32(taddr + c0, regs);
-          tmem_wait_ld();
-          store_columns<32>(p, a, tb * BN + c0, split, regs);
-          __syncwarp();
-        }
-      } else {
-        uint32_t regs[16];
-        tmem_load16(taddr, regs);
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        uint32_t regs[32];
+        tmem_load32(taddr + c0, regs);
         tmem_wait_ld();
-        store_columns<16>(p, a, tb * BN, split, regs);
+        store_columns<32>(p, a, tb * BN + c0, split, regs);
         __syncwarp();
       }
       tcgen05_fence_before();
@@ -932,11 +915,11 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
 }
 
 // ---------------------------------------------------------------------------
-// Weight-streaming kernel for M <= 128 tokens (decode and short prompts).
+// Weight-streaming kernel for 16 < M <= 128 tokens (short prompts, batched decode).
 //
 // The layer is then bound by the one pass over the packed weights, so the
 // kernel is built around that stream: output channels sit on the 128-row MMA
-// axis (operand A), the few tokens on the N axis (BN = 16 .. 128), K is split
+// axis (operand A), the few tokens on the N axis (BN = 32 .. 128), K is split
 // across CTAs so that every SM streams.  As in the two-CTA kernel the streamed
 // operand never returns to shared memory: TMA delivers 64 packed bytes per
 // weight row and k-block, four A-widen warps (one per tensor-memory lane
@@ -951,6 +934,7 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
 // ---------------------------------------------------------------------------
 template <int BN>
 struct Stream {
+  static_assert(BN == 32 || BN == 64 || BN == 128, "token tile");
   static constexpr int kStages = BN <= 64 ? 6 : 4;       // A slots in tensor memory = token stages in shared memory
   static constexpr int kPackedStages = 6;
   static constexpr int kPackedA = kBM * kPackedRow;      // 8 KB of weights
@@ -1165,25 +1149,16 @@ w4a4_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
         // this split's partial sums, token-major [BN][128] int32, over the int8 token stages
         // (every MMA that read them has completed)
         const uint32_t dst = wide_base + uint32_t(e * 32 + lane) * 4u;
-        if constexpr (BN >= 32) {
 #pragma unroll 1
-          for (int c0 = 0; c0 < BN; c0 += 32) {
-            uint32_t regs[32];
-            tmem_load32(taddr + uint32_t(c0), regs);
-            tmem_wait_ld();
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              asm volatile("st.shared.b32 [%0], %1;" ::"r"(dst + uint32_t(c0 + j) * 512u), "r"(regs[j]) : "memory");
-          }
-        } else {
-          uint32_t regs[16];
-          tmem_load16(taddr, regs);
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          uint32_t regs[32];
+          tmem_load32(taddr + uint32_t(c0), regs);
           tmem_wait_ld();
 #pragma unroll
-          for (int j = 0; j < 16; ++j)
-            asm volatile("st.shared.b32 [%0], %1;" ::"r"(dst + uint32_t(j) * 512u), "r"(regs[j]) : "memory");
+          for (int j = 0; j < 32; ++j)
+            asm volatile("st.shared.b32 [%0], %1;" ::"r"(dst + uint32_t(c0 + j) * 512u), "r"(regs[j]) : "memory");
         }
-      } else if constexpr (BN >= 32) {
+      } else {
 #pragma unroll 1
         for (int c0 = 0; c0 < BN; c0 += 32) {
           uint32_t regs[32];
@@ -1192,12 +1167,6 @@ w4a4_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
           store_columns<32>(p, a, tb * BN + c0, split, regs);
           __syncwarp();
         }
-      } else {
-        uint32_t regs[16];
-        tmem_load16(taddr, regs);
-        tmem_wait_ld();
-        store_columns<16>(p, a, tb * BN, split, regs);
-        __syncwarp();
       }
     }
   }
@@ -1742,9 +1711,7 @@ static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq,
   switch (pl.bn) {
     case 256: rc = launch_tile<256>(ma, mb, p, st); break;
     case 128: rc = launch_tile<128>(ma, mb, p, st); break;
-    case 64: rc = launch_tile<64>(ma, mb, p, st); break;
-    case 32: rc = launch_tile<32>(ma, mb, p, st); break;
-    default: rc = launch_tile<16>(ma, mb, p, st); break;
+    default: rc = launch_tile<64>(ma, mb, p, st); break;
   }
   if (rc != SMOOTHROT_OK) return rc;
   if (pl.splits > 1 && !pl.cluster) {
