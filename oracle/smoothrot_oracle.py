@@ -23,6 +23,13 @@ What follows the paper, by passage:
   quantization, group size 128 and clip ratio 0.95 (kv_quantize).
 * Fig. 2 (the feed-forward block): the down-projection input is the gated
   product sigma(gate) (.) up; quant_act_glu takes that edge in one step.
+* Section "Methodology", "two additional Hadamard transformations integrated
+  into the forward pass, as described in [QuaRot]": the paper details the one
+  in front of the down-projection only.  The other sits in front of the
+  attention output projection and, as QuaRot describes it, mixes the heads:
+  (H_heads (x) I_head_dim) / sqrt(heads), the per-head factor
+  (I (x) H_head_dim) being folded into the value projection offline
+  (rotate_heads, rotate_per_head, quant_act_heads).
 
 Floating point: transforms and scales are computed in float64 and rounded once
 to float32; the quantizer decisions (step, division, rounding) are taken in
@@ -380,6 +387,45 @@ def quant_act(X: np.ndarray, pre_x, K: int, clip_a: float = 0.9):
     Lambda^-1 already sits in the producing layer), rotated, quantized per
     token.  Returns (packed [M, K/2] u8, step [M] f32, rotated float32 [M, K])."""
     xr = rotate(X, pre_x, K).astype(np.float32)
+    codes, step = quantize_rows(xr, clip_a)
+    return pack_codes(codes), step, xr
+
+
+def rotate_heads(x: np.ndarray, pre, n_heads: int) -> np.ndarray:
+    """The online transform in front of the attention output projection: a row is the
+    concatenation of n_heads head outputs of head_dim values each, and the heads are mixed
+    by the Walsh-Hadamard matrix,
+        y[m, g * head_dim + e] = sum_h x[m, h * head_dim + e] * pre[h * head_dim + e] * H[h, g] / sqrt(n_heads),
+    i.e. the row times (H_heads (x) I_head_dim) / sqrt(n_heads).  Reading: the paper names
+    this transform only by reference to QuaRot; there it is exact (no diagonal), so `pre` is
+    normally None.  float64."""
+    v = np.asarray(x, dtype=np.float64)
+    assert v.ndim == 2 and v.shape[1] % n_heads == 0
+    if pre is not None:
+        v = v * np.asarray(pre, dtype=np.float64)[None, :]
+    M, K = v.shape
+    H = sylvester(n_heads).astype(np.float64)
+    y = np.einsum("mhe,hg->mge", v.reshape(M, n_heads, K // n_heads), H)
+    return y.reshape(M, K) / np.sqrt(np.float64(n_heads))
+
+
+def rotate_per_head(x: np.ndarray, head_dim: int) -> np.ndarray:
+    """The other factor of the same rotation, (I_heads (x) H_head_dim) / sqrt(head_dim): every
+    head's head_dim values are transformed on their own.  In the model it is folded into the
+    value projection offline (and applied online to queries and keys); here it exists so that
+    the product of the two factors can be checked against the full rotation.  float64."""
+    v = np.asarray(x, dtype=np.float64)
+    assert v.ndim == 2 and v.shape[1] % head_dim == 0
+    M, K = v.shape
+    y = _walsh_last_axis(v.reshape(M, K // head_dim, head_dim))
+    return y.reshape(M, K) / np.sqrt(np.float64(head_dim))
+
+
+def quant_act_heads(X: np.ndarray, pre_x, n_heads: int, clip_a: float = 0.9):
+    """Online activation path in front of the attention output projection: rotate_heads, then
+    the per-token symmetric quantizer of quant_act.  Returns (packed [M, K/2] u8, step [M] f32,
+    rotated float32 [M, K])."""
+    xr = rotate_heads(X, pre_x, n_heads).astype(np.float32)
     codes, step = quantize_rows(xr, clip_a)
     return pack_codes(codes), step, xr
 
