@@ -136,6 +136,24 @@ int smoothrot_quant_act(const void* X_f16, int64_t M, int64_t K, int64_t ldx,
                         uint8_t* Xq_out, float* dx_out, void* stream);
 
 /*
+ * Online activation path in front of the attention output projection.  Methodology section: "two
+ * additional Hadamard transformations integrated into the forward pass, as described in [QuaRot]";
+ * the paper spells out only the one before the down-projection (smoothrot_quant_act).  The other
+ * one, as QuaRot describes it, mixes the heads of the attention output: a row of X is the
+ * concatenation of n_heads head outputs of head_dim values, and
+ *     x^[m][g * head_dim + e] = sum_h X[m][h * head_dim + e] * pre[h * head_dim + e] * H[h][g] / sqrt(n_heads)
+ * with H the Sylvester matrix of order n_heads, i.e. the row times (H_heads (x) I_head_dim) /
+ * sqrt(n_heads); the per-head factor (I (x) H_head_dim) of the full rotation is folded into the
+ * value projection offline.  The transform is exact in the paper's setting, so `pre` is normally
+ * NULL.  dx and the codes follow from x^ exactly as in smoothrot_quant_act.
+ * X is [M x ldx] fp16 with ldx >= K = n_heads * head_dim, Xq_out [M x K/2] bytes, dx_out [M] fp32.
+ * Supported: n_heads in {8, 16, 32, 64}, head_dim in {64, 128, 256} (else SMOOTHROT_UNSUPPORTED_K).
+ */
+int smoothrot_quant_act_heads(const void* X_f16, int64_t M, int64_t n_heads, int64_t head_dim, int64_t ldx,
+                              const float* pre, float clip_a,
+                              uint8_t* Xq_out, float* dx_out, void* stream);
+
+/*
  * The online activation path fed directly by the gated linear unit (Fig. 2: the edge
  * "sigma(gate) (.) up -> hadamard -> quantize" in front of the down-projection; Methodology
  * section: Lambda^-1 is absorbed into the up-projection because the gated product is
@@ -229,11 +247,15 @@ size_t smoothrot_workspace_bytes(int64_t M, int64_t N, int64_t K);
  * Test exports: values the fused kernels never write to memory.
  *   smoothrot_debug_hadamard: Y[m][:] = (X[m][:] * pre) H / sqrt(K) as fp32
  *     [M x K], the rotation alone (Methodology section).
+ *   smoothrot_debug_hadamard_heads: the same for the head-mixing transform of
+ *     smoothrot_quant_act_heads, Y [M x n_heads * head_dim] fp32.
  *   smoothrot_debug_gemm_i32: the int32 accumulators acc [M x N] of
- *     smoothrot_linear, computed by the same tensor-core kernel.
+ *     smoothrot_linear, computed by the same kernels.
  */
 int smoothrot_debug_hadamard(const void* X_f16, int64_t M, int64_t K, int64_t ldx,
                              const float* pre, float* Y_f32, void* stream);
+int smoothrot_debug_hadamard_heads(const void* X_f16, int64_t M, int64_t n_heads, int64_t head_dim,
+                                   int64_t ldx, const float* pre, float* Y_f32, void* stream);
 int smoothrot_debug_gemm_i32(const uint8_t* Xq, int64_t M, const uint8_t* Wq, int64_t N,
                              int64_t K, int32_t* acc,
                              void* workspace, size_t workspace_bytes, void* stream);

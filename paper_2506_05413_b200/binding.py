@@ -27,12 +27,14 @@ SIGNATURES = {
     "smoothrot_fuse_weights_search": (_int, [_vp, _i64, _i64, _i64, _vp, _f32, _int, _vp, _vp, _vp, _vp, _sz, _vp]),
     "smoothrot_quant_act": (_int, [_vp, _i64, _i64, _i64, _vp, _f32, _vp, _vp, _vp]),
     "smoothrot_quant_act_glu": (_int, [_vp, _vp, _i64, _i64, _i64, _i64, _vp, _f32, _vp, _vp, _vp]),
+    "smoothrot_quant_act_heads": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _f32, _vp, _vp, _vp]),
     "smoothrot_kv_quant": (_int, [_vp, _i64, _i64, _i64, _f32, _vp, _vp, _vp, _vp]),
     "smoothrot_kv_dequant": (_int, [_vp, _vp, _vp, _i64, _i64, _vp, _i64, _vp]),
     "smoothrot_linear": (_int, [_vp, _vp, _i64, _vp, _vp, _i64, _i64, _vp, _i64, _vp, _sz, _vp]),
     "smoothrot_linear_static_scratch": (_int, [_vp, _vp, _i64, _vp, _vp, _i64, _i64, _vp, _i64, _vp]),
     "smoothrot_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "smoothrot_debug_hadamard": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp]),
+    "smoothrot_debug_hadamard_heads": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _vp, _vp]),
     "smoothrot_debug_gemm_i32": (_int, [_vp, _i64, _vp, _i64, _i64, _vp, _vp, _sz, _vp]),
     "smoothrot_paley28": (_int, [_vp]),
     "smoothrot_device_status": (_int, [ctypes.POINTER(_int), _int]),
@@ -178,6 +180,19 @@ def quant_act_glu(gate, up, pre, clip_a, Xq_out, dx_out):
                                           _stream()))
 
 
+def quant_act_heads(X, n_heads, pre, clip_a, Xq_out, dx_out):
+    """smoothrot_quant_act_heads: X [M, n_heads * head_dim] fp16, heads mixed by the Walsh-Hadamard matrix,
+    -> Xq_out [M, K/2] u8, dx_out [M] f32."""
+    xp, R, K, ld = _rows(X, torch.float16, "X")
+    if n_heads <= 0 or K % n_heads:
+        raise ValueError("the row length must be a multiple of n_heads")
+    if Xq_out.dtype != torch.uint8 or tuple(Xq_out.shape) != (R, K // 2) or not Xq_out.is_contiguous():
+        raise ValueError(f"Xq_out must be a contiguous uint8 [{R}, {K // 2}] tensor")
+    _check(load().smoothrot_quant_act_heads(xp, R, int(n_heads), K // int(n_heads), ld, _vec(pre, K, "pre"),
+                                            float(clip_a), _ptr(Xq_out, torch.uint8, "Xq_out"),
+                                            _vec(dx_out, R, "dx_out"), _stream()))
+
+
 KV_GROUP = 128
 
 
@@ -254,6 +269,17 @@ def debug_hadamard(X, pre, Y):
         raise ValueError("Y must be a contiguous float32 [M, K] tensor")
     _check(load().smoothrot_debug_hadamard(xp, M, K, ld, _vec(pre, K, "pre"), _ptr(Y, torch.float32, "Y"),
                                            _stream()))
+
+
+def debug_hadamard_heads(X, n_heads, pre, Y):
+    """smoothrot_debug_hadamard_heads: Y [M, K] f32 = (X * pre) (H_heads (x) I) / sqrt(n_heads)."""
+    xp, M, K, ld = _rows(X, torch.float16, "X")
+    if n_heads <= 0 or K % n_heads:
+        raise ValueError("the row length must be a multiple of n_heads")
+    if Y.dtype != torch.float32 or tuple(Y.shape) != (M, K) or not Y.is_contiguous():
+        raise ValueError("Y must be a contiguous float32 [M, K] tensor")
+    _check(load().smoothrot_debug_hadamard_heads(xp, M, int(n_heads), K // int(n_heads), ld, _vec(pre, K, "pre"),
+                                                 _ptr(Y, torch.float32, "Y"), _stream()))
 
 
 def debug_gemm_i32(Xq, Wq, acc, workspace=None):

@@ -56,6 +56,13 @@ def test_host_side_rejections(lib):
     assert q(dummy, 4, 128, 128, None, 1.5, dummy, dummy, None) == -1
     assert q(dummy, 0, 128, 128, None, 0.9, None, None, None) == 0           # empty input is fine
     assert lib.smoothrot_fuse_weights(dummy, 4, 96, 96, None, 1.0, dummy, dummy, None) == -2
+    qh = lib.smoothrot_quant_act_heads
+    assert qh(dummy, 4, 12, 128, 1536, None, 0.9, dummy, dummy, None) == -2      # 12 heads: not a power of two
+    assert qh(dummy, 4, 32, 96, 3072, None, 0.9, dummy, dummy, None) == -2       # head_dim 96
+    assert qh(dummy, 4, 32, 128, 4000, None, 0.9, dummy, dummy, None) == -1      # ldx < K
+    assert qh(dummy, 4, 32, 128, 4096, None, 0.0, dummy, dummy, None) == -1
+    assert qh(odd, 4, 32, 128, 4096, None, 0.9, dummy, dummy, None) == -3
+    assert qh(dummy, 0, 32, 128, 4096, None, 0.9, None, None, None) == 0
     lin = lib.smoothrot_linear
     assert lin(dummy, dummy, 4, dummy, dummy, 8, 100, dummy, 8, None, 0, None) == -2   # K % 128
     assert lin(dummy, dummy, 4, dummy, dummy, 12, 128, dummy, 16, None, 0, None) == -1  # N % 8
