@@ -73,10 +73,7 @@ heads_kernel(const __half* __restrict__ x, int64_t ld, int rows, int head_dim, c
   for (; m < rows; m += row_stride) {
     f32x2 v[NH];
 #pragma unroll
-    for (int h = 0; h < NH; ++h) {
-      const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&raw[h]));
-      v[h] = pack2(f.x, f.y);
-    }
+    for (int h = 0; h < NH; ++h) v[h] = half2_to_f32x2(raw[h]);
     // the next row of this group is on its way during the arithmetic
     const int next = m + row_stride;
     if (next < rows) {

@@ -50,4 +50,19 @@ __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
   return r;
 }
 
+// Two fp16 values (one 32-bit word) to fp32 with the mixed-precision fma of sm_100
+// (x * 1 + 0, exact): it issues on the FMA pipe, where cvt.f32.f16 would queue on the
+// quarter-rate conversion unit.
+__device__ __forceinline__ f32x2 half2_to_f32x2(uint32_t raw) {
+  float lo, hi;
+  asm("{\n\t.reg .b16 l, h, one;\n\t"
+      "mov.b32 {l, h}, %2;\n\t"
+      "mov.b16 one, 0x3C00;\n\t"
+      "fma.rn.f32.f16 %0, l, one, %3;\n\t"
+      "fma.rn.f32.f16 %1, h, one, %3;\n\t}"
+      : "=f"(lo), "=f"(hi)
+      : "r"(raw), "f"(0.0f));
+  return pack2(lo, hi);
+}
+
 }  // namespace smoothrot

@@ -5,7 +5,8 @@
 For every shape (q/o 4096->4096, k/v 4096->1024, gate/up 4096->14336, down 14336->4096) and
 every M in {1, 4, 16, 128, 512, 2048, 8192} it times the two online calls of the layer,
 smoothrot_quant_act and smoothrot_linear, on seeded synthetic activations (random-init
-weights, quantized once by smoothrot_fuse_weights), and prints time, TOP/s and GB/s.
+weights, quantized once by smoothrot_fuse_weights), and prints time, TOP/s and GB/s; for the q/o
+shape also smoothrot_quant_act_heads (32 heads of 128), the transform the o-projection's input takes.
 
 Timing: each call is recorded into a CUDA graph per buffer set and replayed back to back
 between two CUDA events; the buffer sets rotate so that their total size exceeds twice the
@@ -21,6 +22,7 @@ import numpy as np
 from . import synth
 
 L2_BYTES = 126 * 1024 * 1024
+HEADS = 32          # 32 heads of 128: the attention output of the 8B-class models
 
 
 def _time_graphs(torch, graphs, reps):
@@ -73,18 +75,25 @@ def run(reps: int = 30, shapes=None, tokens=None):
                 sr.linear(xq, dx, wq, dw, Y, ws)
                 sets.append((X, xq, dx, wq, dw, Y, ws))
             torch.cuda.synchronize()
-            gq, gl = [], []
+            gq, gl, gh = [], [], []
             for X, xq, dx, wq, dw, Y, ws in sets:
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g):
                     sr.quant_act(X, pre_x, case.clip_a, xq, dx)
                 gq.append(g)
+                if name == "q_o":      # the o-projection's input also has the head-mixing variant
+                    sr.quant_act_heads(X, HEADS, None, case.clip_a, xq, dx)
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g):
+                        sr.quant_act_heads(X, HEADS, None, case.clip_a, xq, dx)
+                    gh.append(g)
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g):
                     sr.linear(xq, dx, wq, dw, Y, ws)
                 gl.append(g)
-            tq = _time_graphs(torch, gq, reps)
             tl = _time_graphs(torch, gl, reps)
+            th = _time_graphs(torch, gh, reps) if gh else None
+            tq = _time_graphs(torch, gq, reps)
             assert sr.device_status() == 0
             ops = 2.0 * M * N * K
             rows.append({
@@ -95,6 +104,9 @@ def run(reps: int = 30, shapes=None, tokens=None):
                 "weight_stream_GBs": 0.5 * N * K / tl / 1e9,
                 "buffer_sets": n_sets,
             })
+            if th is not None:
+                rows[-1]["quant_act_heads_us"] = th * 1e6
+                rows[-1]["quant_act_heads_GBs"] = (2.5 * M * K + 4 * M) / th / 1e9
             del sets, gq, gl
             torch.cuda.empty_cache()
     return rows
@@ -112,10 +124,13 @@ def main():
         for r in rows:
             print(json.dumps(r))
         return
-    print(f"{'shape':8s} {'M':>5s} {'quant us':>9s} {'GB/s':>7s} {'linear us':>10s} {'TOP/s':>8s} {'W GB/s':>8s}")
+    print(f"{'shape':8s} {'M':>5s} {'quant us':>9s} {'GB/s':>7s} {'linear us':>10s} {'TOP/s':>8s} {'W GB/s':>8s}"
+          f" {'heads us':>9s} {'GB/s':>7s}")
     for r in rows:
+        heads = (f" {r['quant_act_heads_us']:9.1f} {r['quant_act_heads_GBs']:7.0f}"
+                 if "quant_act_heads_us" in r else "")
         print(f"{r['shape']:8s} {r['M']:5d} {r['quant_act_us']:9.1f} {r['quant_act_GBs']:7.0f} "
-              f"{r['linear_us']:10.1f} {r['linear_TOPS']:8.1f} {r['weight_stream_GBs']:8.0f}")
+              f"{r['linear_us']:10.1f} {r['linear_TOPS']:8.1f} {r['weight_stream_GBs']:8.0f}{heads}")
 
 
 if __name__ == "__main__":
