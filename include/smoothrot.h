@@ -239,8 +239,12 @@ int smoothrot_kv_quant(const void* X_f16, int64_t rows, int64_t C, int64_t ldx, 
 int smoothrot_kv_dequant(const uint8_t* q, const float* step, const float* zero, int64_t rows,
                          int64_t C, void* Y_f16, int64_t ldy, void* stream);
 
-/* Host. Scratch bytes smoothrot_linear / smoothrot_debug_gemm_i32 need for
- * this shape (0 for shapes that need none). */
+/* Host. Scratch bytes smoothrot_linear / smoothrot_debug_gemm_i32 want for
+ * this shape (0 for shapes that need none).  With M <= 128 a shape that reports
+ * a size cannot run without it (SMOOTHROT_WORKSPACE_TOO_SMALL).  With M >= 256 the
+ * scratch only serves to split K over otherwise idle SMs (few output tiles, long
+ * K): with a smaller or absent workspace the call runs unsplit, slower but with
+ * the same result. */
 size_t smoothrot_workspace_bytes(int64_t M, int64_t N, int64_t K);
 
 /*

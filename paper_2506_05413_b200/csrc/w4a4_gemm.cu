@@ -645,10 +645,12 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t tmem_a_ring = tmem_base + uint32_t(T::kAccCols);
 
-  const int total_tiles = p.tiles_a * p.tiles_b;
+  // a unit of work is (tile, k-split); with k-splits the int32 partial sums go to the workspace
+  const int tiles_ab = p.tiles_a * p.tiles_b;
+  const int total_tiles = tiles_ab * p.splits;
   const int first_tile = blockIdx.x >> 1;
   const int tile_step = gridDim.x >> 1;
-  const int kblocks = p.kblocks;
+  const int kblocks = p.kblocks / p.splits;   // host guarantees divisibility
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (each CTA, own rows)
@@ -656,16 +658,18 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
       uint32_t it = 0;
       bool ok = true;
       for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
-        const int ta = tile % p.tiles_a;
-        const int tb = tile / p.tiles_a;
+        const int ta = (tile % tiles_ab) % p.tiles_a;
+        const int tb = (tile % tiles_ab) / p.tiles_a;
+        const int kb0 = (tile / tiles_ab) * kblocks;
         for (int kb = 0; kb < kblocks; ++kb, ++it) {
           const int s = it % T::kPackedStages;
           const uint32_t ph = (it / T::kPackedStages) & 1u;
           if (!mbar_wait(pk_empty(s), ph ^ 1u, abort_flag, kSiteProducer)) { ok = false; break; }
           mbar_expect_tx(pk_full(s), uint32_t(T::kPackedA + T::kPackedB));
           const uint32_t dst = packed_base + s * T::kPackedStageBytes;
-          tma_load_2d(dst, &map_a, pk_full(s), kb * kPackedRow, ta * 256 + int(rank) * kBM);
-          tma_load_2d(dst + T::kPackedA, &map_b, pk_full(s), kb * kPackedRow, tb * T::kBN + int(rank) * T::kHalfN);
+          tma_load_2d(dst, &map_a, pk_full(s), (kb0 + kb) * kPackedRow, ta * 256 + int(rank) * kBM);
+          tma_load_2d(dst + T::kPackedA, &map_b, pk_full(s), (kb0 + kb) * kPackedRow,
+                      tb * T::kBN + int(rank) * T::kHalfN);
         }
       }
     }
@@ -811,8 +815,9 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
     const uint32_t dw_warp = dw_base + uint32_t(q) * uint32_t(T::kBN * 4);
     uint32_t local_tile = 0;
     for (int tile = first_tile; tile < total_tiles; tile += tile_step, ++local_tile) {
-      const int ta = tile % p.tiles_a;
-      const int tb = tile / p.tiles_a;
+      const int ta = (tile % tiles_ab) % p.tiles_a;
+      const int tb = (tile % tiles_ab) / p.tiles_a;
+      const int split = tile / tiles_ab;
       const int row0 = ta * 256 + int(rank) * kBM + q * 32;
       const int a = row0 + lane;
       float sx = 0.0f;
@@ -883,13 +888,13 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
         }
         if (lane == 0) tma_store_commit();
       } else {
-        // test export of the int32 accumulators: plain stores
+        // int32 accumulators (partial sums of a k-split, or the test export): plain stores
 #pragma unroll 1
         for (int c0 = 0; c0 < T::kBN; c0 += 32) {
           uint32_t regs[32];
           tmem_load32(taddr + uint32_t(c0), regs);
           tmem_wait_ld();
-          store_columns<32>(p, a, tb * T::kBN + c0, 0, regs);
+          store_columns<32>(p, a, tb * T::kBN + c0, split, regs);
           __syncwarp();
         }
         tcgen05_fence_before();
@@ -1493,6 +1498,8 @@ static int sm_count() {
   return cached;
 }
 
+constexpr int kPairSplitMinBlocks = 32;   // k-blocks per split below which the extra pass over the partial sums costs more than it saves
+
 static Plan make_plan(int64_t M, int64_t N, int64_t K) {
   Plan pl{};
   const int kblocks = int(K / kWideRow);
@@ -1510,6 +1517,10 @@ static Plan make_plan(int64_t M, int64_t N, int64_t K) {
     pl.pair = M >= 256 && N >= 256;
     pl.bn = (N >= 256) ? 256 : (N > 64 ? 128 : 64);
     pl.splits = 1;
+    // Few tiles and a long K: two k-splits per tile put twice as many SM pairs to work; the partial
+    // sums take the workspace path.
+    if (pl.pair && 2 * pair_tiles <= sm_count() / 2 && kblocks % 2 == 0 && kblocks / 2 >= kPairSplitMinBlocks)
+      pl.splits = 2;
     return pl;
   }
   pl.swapped = true;
@@ -1624,6 +1635,16 @@ static int launch_tile(const CUtensorMap& ma, const CUtensorMap& mb, const Param
   return launch_status();
 }
 
+static int launch_splitk_reduce(const void* workspace, int splits, int64_t M, int64_t N, const float* dx,
+                                const float* dw, __half* Y, int64_t ldy, int32_t* acc_out, cudaStream_t st) {
+  const int64_t total = M * (N / 8);
+  const int threads = 256;
+  splitk_reduce_kernel<<<unsigned((total + threads - 1) / threads), threads, 0, st>>>(
+      static_cast<const int32_t*>(workspace), splits, int(M), int(N), dx, dw, Y, ldy, acc_out);
+  count_launch();
+  return launch_status();
+}
+
 static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq, const float* dw, int64_t N,
                int64_t K, __half* Y, int64_t ldy, int32_t* acc_out, void* workspace, size_t workspace_bytes,
                cudaStream_t st) {
@@ -1641,8 +1662,13 @@ static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq,
     if (acc_out == nullptr) return SMOOTHROT_INVALID_ARG;
     if (!aligned16(acc_out)) return SMOOTHROT_BAD_ALIGNMENT;
   }
-  const Plan pl = make_plan(M, N, K);
-  const size_t need = (pl.splits > 1 && !pl.cluster) ? size_t(pl.splits) * size_t(M) * size_t(N) * sizeof(int32_t) : 0;
+  Plan pl = make_plan(M, N, K);
+  size_t need = (pl.splits > 1 && !pl.cluster) ? size_t(pl.splits) * size_t(M) * size_t(N) * sizeof(int32_t) : 0;
+  if (pl.pair && need > 0 && (workspace == nullptr || workspace_bytes < need)) {
+    // the two-CTA kernel splits K only to fill idle SM pairs: without the workspace it runs unsplit
+    pl.splits = 1;
+    need = 0;
+  }
   if (need > 0 && (workspace == nullptr || workspace_bytes < need)) return SMOOTHROT_WORKSPACE_TOO_SMALL;
   if (need > 0 && !aligned16(workspace)) return SMOOTHROT_BAD_ALIGNMENT;
 
@@ -1691,12 +1717,14 @@ static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq,
     auto kern = w4a4_gemm_pair_tmem_kernel;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PairT::kSmemBytes) != cudaSuccess)
       return SMOOTHROT_CUDA_ERROR;
-    const int total = p.tiles_a * p.tiles_b;
+    const int total = p.tiles_a * p.tiles_b * pl.splits;
     const int pairs = sm_count() / 2;
     const int grid = 2 * (total < pairs ? total : pairs);
     kern<<<grid, PairT::kThreads, PairT::kSmemBytes, st>>>(ma, mb, my, p);
     count_launch();
-    return launch_status();
+    const int rc = launch_status();
+    if (rc != SMOOTHROT_OK || pl.splits == 1) return rc;
+    return launch_splitk_reduce(workspace, pl.splits, M, N, dx, dw, Y, ldy, acc_out, st);
   }
   if (!make_map(&ma, a_ptr, p.rows_a, K, kBM) || !make_map(&mb, b_ptr, p.rows_b, K, pl.bn))
     return SMOOTHROT_CUDA_ERROR;
@@ -1714,14 +1742,7 @@ static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq,
     default: rc = launch_tile<64>(ma, mb, p, st); break;
   }
   if (rc != SMOOTHROT_OK) return rc;
-  if (pl.splits > 1 && !pl.cluster) {
-    const int64_t total = M * (N / 8);
-    const int threads = 256;
-    splitk_reduce_kernel<<<unsigned((total + threads - 1) / threads), threads, 0, st>>>(
-        static_cast<const int32_t*>(workspace), pl.splits, int(M), int(N), dx, dw, Y, ldy, acc_out);
-    count_launch();
-    rc = launch_status();
-  }
+  if (pl.splits > 1 && !pl.cluster) rc = launch_splitk_reduce(workspace, pl.splits, M, N, dx, dw, Y, ldy, acc_out, st);
   return rc;
 }
 
@@ -1767,8 +1788,12 @@ int smoothrot_linear_static_scratch(const uint8_t* Xq, const float* dx, int64_t 
                                     void* stream) {
   using namespace smoothrot::gemm;
   if (M > 0 && N > 0 && Y_f16 == nullptr) return SMOOTHROT_INVALID_ARG;
-  const size_t need = smoothrot_workspace_bytes(M, N, K);
-  if (need > kStaticScratchBytes) return SMOOTHROT_STATIC_SCRATCH_EXCEEDED;
+  size_t need = smoothrot_workspace_bytes(M, N, K);
+  if (need > kStaticScratchBytes) {
+    // prefill shapes split K only as an optimisation and run without scratch memory as well
+    if (M <= 0 || N <= 0 || K <= 0 || !make_plan(M, N, K).pair) return SMOOTHROT_STATIC_SCRATCH_EXCEEDED;
+    need = 0;
+  }
   void* scratch = nullptr;
   if (need > 0) {
     const int rc = static_scratch_address(&scratch);

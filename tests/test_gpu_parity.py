@@ -179,6 +179,8 @@ GEMM_SHAPES = [
     (256, 256, 128),     # one two-CTA pair tile
     (600, 776, 512),     # two-CTA tiles, ragged in both directions
     (512, 1024, 14336),  # long K
+    (300, 2560, 8192),   # two-CTA tiles with two k-splits through the workspace
+    (520, 2568, 8192),   # ... ragged in both directions
     (17, 1000, 1024),    # streaming kernel, 2 k-splits added up inside a cluster, ragged channels
     (20, 520, 4096),     # 8 k-splits in a cluster
     (40, 136, 2048),     # 64-token tile, 4 k-splits in a cluster
@@ -213,7 +215,7 @@ def test_gemm_extreme_codes(gu):
 @pytest.mark.parametrize("M,N,K", [(64, 256, 128), (3, 1024, 4096), (200, 264, 512), (130, 520, 4096),
                                    (300, 520, 640), (1024, 768, 4096), (16, 1000, 2048), (128, 520, 1024),
                                    (24, 256, 16384), (4, 1000, 14336), (1, 4096, 4096), (6, 1024, 4096), (16, 520, 14336),
-                                   (12, 4104, 2048), (32, 1024, 4096)])
+                                   (12, 4104, 2048), (32, 1024, 4096), (300, 2568, 8192)])
 def test_linear_output_matches_oracle_on_gpu_codes(gu, M, N, K):
     rng = np.random.default_rng(M + N + K)
     xq = orc.pack_codes(synth.random_codes(M, M, K))
@@ -224,6 +226,31 @@ def test_linear_output_matches_oracle_on_gpu_codes(gu, M, N, K):
     want = orc.linear(xq, dx, wq, dw)
     assert np.isfinite(got.astype(np.float32)).all()
     assert gu.rowwise_rel(got, want) <= TOL_OUT
+
+
+def test_prefill_k_split_is_optional_and_changes_nothing(gu):
+    """For M >= 256 the workspace only lets the two-CTA kernel split K over idle SM pairs: without
+    it the call runs unsplit and, the sums being integers, returns the same fp16 outputs."""
+    import torch
+    from paper_2506_05413_b200 import binding as sr
+    M, N, K = 300, 2568, 8192
+    assert sr.workspace_bytes(M, N, K) > 0
+    rng = np.random.default_rng(5)
+    xq = gu.dev(orc.pack_codes(synth.random_codes(1, M, K)))
+    wq = gu.dev(orc.pack_codes(synth.random_codes(2, N, K)))
+    dx = gu.dev(rng.uniform(0.01, 0.3, M).astype(np.float32))
+    dw = gu.dev(rng.uniform(1e-4, 4e-3, N).astype(np.float32))
+    ws = torch.empty(sr.workspace_bytes(M, N, K), dtype=torch.uint8, device=gu.DEV)
+    Y_split = torch.full((M, N), float("nan"), dtype=torch.float16, device=gu.DEV)
+    Y_plain = torch.full((M, N), float("nan"), dtype=torch.float16, device=gu.DEV)
+    Y_short = torch.full((M, N), float("nan"), dtype=torch.float16, device=gu.DEV)
+    sr.linear(xq, dx, wq, dw, Y_split, ws)
+    sr.linear(xq, dx, wq, dw, Y_plain, None)
+    sr.linear(xq, dx, wq, dw, Y_short, ws[:1024])
+    torch.cuda.synchronize()
+    assert sr.device_status() == 0
+    assert torch.equal(Y_split, Y_plain) and torch.equal(Y_split, Y_short)
+    assert bool(torch.isfinite(Y_split).all())
 
 
 # ------------------------------------------------------------- whole layer
