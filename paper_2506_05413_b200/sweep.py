@@ -1,6 +1,7 @@
 """Token-count sweep over the linear shapes of one LLaMA-3.1-8B-shaped decoder block.
 
-    python -m paper_2506_05413_b200.sweep [--reps 30] [--json]
+    python -m paper_2506_05413_b200.sweep [--reps 30] [--json] [--shapes ...] [--tokens ...]
+    python -m paper_2506_05413_b200.sweep --kv        # the KV-cache codec instead
 
 For every shape (q/o 4096->4096, k/v 4096->1024, gate/up 4096->14336, down 14336->4096) and
 every M in {1, 4, 16, 128, 512, 2048, 8192} it times the two online calls of the layer,
@@ -112,13 +113,56 @@ def run(reps: int = 30, shapes=None, tokens=None):
     return rows
 
 
+def run_kv(reps: int = 30, rows: int = 65536, width: int = 1024):
+    """Times the KV-cache codec (smoothrot_kv_quant / smoothrot_kv_dequant) on `rows` cache rows of
+    `width` values (8 KV heads of 128), two buffer sets of seeded N(0,1) values, each larger than L2."""
+    import torch
+    from . import binding as sr
+
+    sr.load()
+    dev = "cuda:0"
+    rng = np.random.default_rng(7)
+    host = torch.from_numpy(rng.standard_normal((rows, width), dtype=np.float32).astype(np.float16))
+    sets = []
+    for _ in range(2):
+        X = host.to(dev)
+        q = torch.empty((rows, width // 2), dtype=torch.uint8, device=dev)
+        step = torch.empty((rows, width // 128), dtype=torch.float32, device=dev)
+        zero = torch.empty_like(step)
+        Y = torch.empty_like(X)
+        sr.kv_quant(X, 0.95, q, step, zero)
+        sr.kv_dequant(q, step, zero, Y)
+        sets.append((X, q, step, zero, Y))
+    torch.cuda.synchronize()
+    gq, gd = [], []
+    for X, q, step, zero, Y in sets:
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            sr.kv_quant(X, 0.95, q, step, zero)
+        gq.append(g)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            sr.kv_dequant(q, step, zero, Y)
+        gd.append(g)
+    tq = _time_graphs(torch, gq, reps)
+    td = _time_graphs(torch, gd, reps)
+    n = rows * width
+    bytes_per_call = n * (2 + 0.5 + 8 / 128)
+    return {"rows": rows, "width": width, "kv_quant_us": tq * 1e6, "kv_quant_GBs": bytes_per_call / tq / 1e9,
+            "kv_dequant_us": td * 1e6, "kv_dequant_GBs": bytes_per_call / td / 1e9}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--reps", type=int, default=30)
     ap.add_argument("--json", action="store_true")
     ap.add_argument("--shapes", nargs="*")
     ap.add_argument("--tokens", nargs="*", type=int)
+    ap.add_argument("--kv", action="store_true", help="time the KV-cache codec instead of the linear shapes")
     args = ap.parse_args()
+    if args.kv:
+        print(json.dumps(run_kv(args.reps)))
+        return
     rows = run(args.reps, args.shapes, args.tokens)
     if args.json:
         for r in rows:
