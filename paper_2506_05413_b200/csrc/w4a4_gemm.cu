@@ -27,9 +27,9 @@
 // the 128-row MMA axis, tokens on the N axis) and K is split across CTAs;
 // the int32 partial sums are added inside a thread-block cluster, or go to the
 // caller's workspace where a second kernel adds them and dequantizes.
-// For M <= 16 tokens none of this machinery pays: a small kernel streams the
-// weights with plain loads and forms the products with the warp-level integer
-// MMA (see the decode kernel near the end).
+// For up to 32 tokens (64 with small weight matrices) none of this machinery
+// pays: a small kernel streams the weights with plain loads and forms the
+// products with the warp-level integer MMA (see the decode kernel near the end).
 //
 // Every wait on an mbarrier is bounded in wall time; a wait that runs out
 // sets a device status word, raises a CTA-wide abort flag and the kernel
@@ -920,11 +920,13 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
 }
 
 // ---------------------------------------------------------------------------
-// Weight-streaming kernel for 16 < M <= 128 tokens (short prompts, batched decode).
+// Weight-streaming kernel for up to 128 tokens per tile (short prompts, batched decode beyond
+// the reach of the decode kernel).
 //
 // The layer is then bound by the one pass over the packed weights, so the
 // kernel is built around that stream: output channels sit on the 128-row MMA
-// axis (operand A), the few tokens on the N axis (BN = 32 .. 128), K is split
+// axis (operand A), the tokens on the N axis (BN = 128; narrower tiles are supported by the
+// template but lost to this one or to the decode kernel on every shape measured), K is split
 // across CTAs so that every SM streams.  As in the two-CTA kernel the streamed
 // operand never returns to shared memory: TMA delivers 64 packed bytes per
 // weight row and k-block, four A-widen warps (one per tensor-memory lane
@@ -1272,7 +1274,7 @@ splitk_reduce_kernel(const int32_t* __restrict__ part, int splits, int M, int N,
 }
 
 // ---------------------------------------------------------------------------
-// Decode kernel for M <= 16 tokens.
+// Decode kernel for few tokens (M <= 8 * NT, NT = 1, 2, 4, 8 token tiles).
 //
 // With a handful of tokens the layer is one pass over the packed weights and nothing else,
 // and the tensor-memory kernels spend more time on their set-up (cluster launch, tensor-memory
@@ -1477,7 +1479,7 @@ static int launch_decode(const uint8_t* Xq, const uint8_t* Wq, int M, int N, int
 // Host side
 // ---------------------------------------------------------------------------
 struct Plan {
-  bool gemv;      // M <= 16: the decode kernel
+  bool gemv;      // few tokens: the decode kernel
   bool swapped;
   bool pair;      // two-CTA kernel, 256 x 256 pair tiles
   bool cluster;   // the k-splits of a tile form a cluster and add up in shared memory (no workspace)
@@ -1503,7 +1505,9 @@ constexpr int kPairSplitMinBlocks = 32;   // k-blocks per split below which the 
 static Plan make_plan(int64_t M, int64_t N, int64_t K) {
   Plan pl{};
   const int kblocks = int(K / kWideRow);
-  if (M <= 16) {                   // the decode kernel: no tiles, no k-splits, no workspace
+  // The decode kernel (no tiles, no k-splits, no workspace) up to 32 tokens, and up to 64 where the
+  // weights are small enough that the tokens' codes, which every CTA reads from L2, do not dominate.
+  if (M <= 32 || (M <= 64 && N * K <= (int64_t(1) << 25))) {
     pl.gemv = true;
     pl.splits = 1;
     return pl;
@@ -1524,10 +1528,9 @@ static Plan make_plan(int64_t M, int64_t N, int64_t K) {
     return pl;
   }
   pl.swapped = true;
-  pl.bn = M <= 32 ? 32 : (M <= 64 ? 64 : 128);
+  pl.bn = 128;   // narrower token tiles were slower than this one on every shape they served
   const int tiles = int((N + kBM - 1) / kBM) * int((M + pl.bn - 1) / pl.bn);
-  // two CTAs of the streaming kernel share an SM, except with the 128-token tile
-  const int slots = (pl.bn <= 64 ? 2 : 1) * sm_count();
+  const int slots = sm_count();   // one CTA of the streaming kernel per SM
   int want = (slots + tiles - 1) / tiles;
   if (want < 1) want = 1;
   // Workspace path: the largest divisor of kblocks that does not exceed `want` and leaves >= 4
@@ -1680,7 +1683,9 @@ static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq,
     const int m = int(M), n = int(N), k = int(K);
 #define SR_DECODE(NT, RG, U, W, P) launch_decode<NT, RG, U, W, P>(Xq, Wq, m, n, k, dx, dw, Y, ldy, out32, st)
     if (M <= 8) return K > 4096 ? SR_DECODE(1, 1, 4, 8, true) : SR_DECODE(1, 1, 4, 8, false);
-    return K > 4096 ? SR_DECODE(2, 2, 2, 16, true) : SR_DECODE(2, 1, 4, 8, false);
+    if (M <= 16) return K > 4096 ? SR_DECODE(2, 2, 2, 16, true) : SR_DECODE(2, 1, 4, 8, false);
+    if (M <= 32) return N >= 8192 ? SR_DECODE(4, 2, 1, 8, true) : SR_DECODE(4, 1, 2, 8, false);
+    return SR_DECODE(8, 1, 1, 8, false);
 #undef SR_DECODE
   }
   Params p{};
@@ -1730,11 +1735,7 @@ static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq,
     return SMOOTHROT_CUDA_ERROR;
   int rc;
   if (pl.swapped) {
-    switch (pl.bn) {
-      case 128: rc = launch_stream<128>(ma, mb, p, st); break;
-      case 64: rc = launch_stream<64>(ma, mb, p, st); break;
-      default: rc = launch_stream<32>(ma, mb, p, st); break;
-    }
+    rc = launch_stream<128>(ma, mb, p, st);
   } else
   switch (pl.bn) {
     case 256: rc = launch_tile<256>(ma, mb, p, st); break;

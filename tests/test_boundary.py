@@ -70,12 +70,12 @@ def test_host_side_rejections(lib):
     assert lin(odd, dummy, 4, dummy, dummy, 8, 128, dummy, 8, None, 0, None) == -3
     assert lin(dummy, dummy, 0, dummy, dummy, 8, 128, dummy, 8, None, 0, None) == 0
     # a shape that splits K needs a workspace
-    need = lib.smoothrot_workspace_bytes(24, 256, 16384)
+    need = lib.smoothrot_workspace_bytes(100, 256, 16384)
     assert need > 0 and need % (4 * 256 * 4) == 0
-    assert lin(dummy, dummy, 24, dummy, dummy, 256, 16384, dummy, 256, None, 0, None) == -4
-    assert lin(dummy, dummy, 24, dummy, dummy, 256, 16384, dummy, 256, dummy, need - 1, None) == -4
-    assert lib.smoothrot_workspace_bytes(32, 1024, 4096) == 0    # k-splits reduced inside a cluster
-    assert lib.smoothrot_workspace_bytes(16, 256, 16384) == 0    # M <= 16: the decode kernel splits K inside a CTA
+    assert lin(dummy, dummy, 100, dummy, dummy, 256, 16384, dummy, 256, None, 0, None) == -4
+    assert lin(dummy, dummy, 100, dummy, dummy, 256, 16384, dummy, 256, dummy, need - 1, None) == -4
+    assert lib.smoothrot_workspace_bytes(128, 1024, 4096) == 0   # k-splits reduced inside a cluster
+    assert lib.smoothrot_workspace_bytes(32, 256, 16384) == 0    # few tokens: the decode kernel splits K inside a CTA
     assert lib.smoothrot_workspace_bytes(2048, 6144, 4096) == 0
     cal = lib.smoothrot_calibrate
     assert cal(dummy, 4, 128, 128, None, 0, 0, 0.5, 1, dummy, dummy, None, None, None, None) == -1  # finalize, no W

@@ -154,9 +154,9 @@ def test_config3_full_size(env):
 
 @pytest.mark.parametrize("shape", [name for name, _, _ in synth.BLOCK_SHAPES])
 def test_token_sweep_decode_shapes_in_full(env, shape):
-    """configs[4]: M = 1, 4, 16, 32, 128 for each linear shape of the block, every output checked."""
+    """configs[4]: M = 1, 4, 16, 32, 64, 128 for each linear shape of the block, every output checked."""
     torch, sr = env
-    for M in (1, 4, 16, 32, 128):
+    for M in (1, 4, 16, 32, 64, 128):
         case = synth.config4(shape, M)
         g = _run_layer(torch, sr, case)
         xq, wq = g["xq"].cpu().numpy(), g["wq"].cpu().numpy()

@@ -152,7 +152,7 @@ def test_calibration_matches_oracle(gu, K, T, N, batches):
 # --------------------------------------------------------------------- GEMM
 GEMM_SHAPES = [
     (64, 256, 128),      # config 0
-    # M <= 16: the decode kernel (plain loads, warp-level integer MMA, K split between the warps of a CTA)
+    # few tokens: the decode kernel (plain loads, warp-level integer MMA, K split between the warps of a CTA)
     (1, 1024, 4096),
     (4, 4096, 4096),
     (2, 1000, 1024),     # ragged channels (N % 16 == 8)
@@ -168,27 +168,36 @@ GEMM_SHAPES = [
     (16, 1000, 8192),
     (13, 520, 4224),     # long rows with a partial last batch
     (8, 256, 16384),
-    # the streaming kernel
-    (17, 64, 256),       # 32-wide token tile
-    (33, 72, 384),       # 64-wide token tile
-    (100, 264, 256),     # 128-wide token tile, swapped
-    (128, 64, 128),      # prefill, BN = 64
-    (130, 136, 640),     # BN = 128, ragged both ways
-    (300, 520, 1152),    # BN = 256, several tiles and a ragged tail
-    (257, 8, 128),
-    (256, 256, 128),     # one two-CTA pair tile
-    (600, 776, 512),     # two-CTA tiles, ragged in both directions
-    (512, 1024, 14336),  # long K
-    (300, 2560, 8192),   # two-CTA tiles with two k-splits through the workspace
-    (520, 2568, 8192),   # ... ragged in both directions
-    (17, 1000, 1024),    # streaming kernel, 2 k-splits added up inside a cluster, ragged channels
-    (20, 520, 4096),     # 8 k-splits in a cluster
-    (40, 136, 2048),     # 64-token tile, 4 k-splits in a cluster
-    (128, 1024, 4096),   # 128-token tile, cluster
-    (24, 256, 16384),    # few channels, long K: k-splits through the workspace
+    (17, 64, 256),       # four token tiles
+    (20, 520, 4096),
+    (24, 256, 16384),
+    (32, 8200, 512),     # four token tiles, many channels: two row groups per CTA, double-buffered
+    (25, 8456, 1152),
+    (33, 72, 384),       # eight token tiles
+    (40, 136, 2048),
+    (64, 1000, 4096),
+    (50, 264, 14336),
+    # the streaming kernel (128-token tiles)
+    (64, 8200, 4096),    # 64 tokens, but too many weights for the decode kernel
+    (100, 264, 256),
+    (128, 64, 128),
+    (70, 1000, 1024),    # 2 k-splits added up inside a cluster, ragged channels
+    (80, 520, 4096),     # 8 k-splits in a cluster
+    (128, 1024, 4096),
+    (100, 256, 16384),   # few channels, long K: k-splits through the workspace
     (128, 256, 8192),
     (300, 1024, 2048),   # 3 token tiles of the streaming kernel, ragged
     (512, 520, 1024),
+    (512, 1024, 14336),  # long K
+    # one CTA per SM, both operands through shared memory
+    (130, 136, 640),     # BN = 128, ragged both ways
+    (300, 520, 1152),    # BN = 256, several tiles and a ragged tail
+    (257, 8, 128),
+    # the two-CTA kernel
+    (256, 256, 128),     # one pair tile
+    (600, 776, 512),     # ragged in both directions
+    (300, 2560, 8192),   # two k-splits through the workspace
+    (520, 2568, 8192),   # ... ragged in both directions
 ]
 
 
@@ -214,7 +223,8 @@ def test_gemm_extreme_codes(gu):
 
 @pytest.mark.parametrize("M,N,K", [(64, 256, 128), (3, 1024, 4096), (200, 264, 512), (130, 520, 4096),
                                    (300, 520, 640), (1024, 768, 4096), (16, 1000, 2048), (128, 520, 1024),
-                                   (24, 256, 16384), (4, 1000, 14336), (1, 4096, 4096), (6, 1024, 4096), (16, 520, 14336),
+                                   (100, 256, 16384), (4, 1000, 14336), (1, 4096, 4096), (6, 1024, 4096), (16, 520, 14336),
+                                   (30, 8200, 1024), (64, 520, 4096), (64, 8200, 4096),
                                    (12, 4104, 2048), (32, 1024, 4096), (300, 2568, 8192)])
 def test_linear_output_matches_oracle_on_gpu_codes(gu, M, N, K):
     rng = np.random.default_rng(M + N + K)
