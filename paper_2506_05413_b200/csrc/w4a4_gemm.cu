@@ -1512,14 +1512,17 @@ static Plan make_plan(int64_t M, int64_t N, int64_t K) {
     pl.splits = 1;
     return pl;
   }
-  // Up to 512 tokens the two-CTA kernel's 256 x 256 tiles can leave most SM pairs idle (few output
-  // channels); the streaming kernel with 128-token tiles and k-splits then fills the machine better.
+  // The two-CTA kernel works on 256 x 256 tiles, one per SM pair.  Up to 256 tokens (one row of
+  // tiles) it is taken when the output channels alone fill more than half of the pairs, and the
+  // streaming kernel with 128-token tiles and k-splits otherwise; up to 512 tokens the streaming
+  // kernel still wins when the tiles are very few.
   const int64_t pair_tiles = ((M + 255) / 256) * ((N + 255) / 256);
-  const bool few_pair_tiles = M <= 512 && 16 * pair_tiles <= sm_count();
-  if (M > 128 && !few_pair_tiles) {
+  const bool to_stream = M <= 256 ? !(N >= 256 && 4 * pair_tiles > sm_count())
+                                  : (M <= 512 && 16 * pair_tiles <= sm_count());
+  if (!to_stream) {
     pl.swapped = false;
-    pl.pair = M >= 256 && N >= 256;
-    pl.bn = (N >= 256) ? 256 : (N > 64 ? 128 : 64);
+    pl.pair = N >= 256;
+    pl.bn = N > 64 ? 128 : 64;   // of the one-CTA kernel that serves N < 256
     pl.splits = 1;
     // Few tiles and a long K: two k-splits per tile put twice as many SM pairs to work; the partial
     // sums take the workspace path.
@@ -1737,11 +1740,7 @@ static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq,
   if (pl.swapped) {
     rc = launch_stream<128>(ma, mb, p, st);
   } else
-  switch (pl.bn) {
-    case 256: rc = launch_tile<256>(ma, mb, p, st); break;
-    case 128: rc = launch_tile<128>(ma, mb, p, st); break;
-    default: rc = launch_tile<64>(ma, mb, p, st); break;
-  }
+  rc = pl.bn == 128 ? launch_tile<128>(ma, mb, p, st) : launch_tile<64>(ma, mb, p, st);
   if (rc != SMOOTHROT_OK) return rc;
   if (pl.splits > 1 && !pl.cluster) rc = launch_splitk_reduce(workspace, pl.splits, M, N, dx, dw, Y, ldy, acc_out, st);
   return rc;

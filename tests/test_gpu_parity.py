@@ -189,12 +189,16 @@ GEMM_SHAPES = [
     (300, 1024, 2048),   # 3 token tiles of the streaming kernel, ragged
     (512, 520, 1024),
     (512, 1024, 14336),  # long K
-    # one CTA per SM, both operands through shared memory
-    (130, 136, 640),     # BN = 128, ragged both ways
-    (300, 520, 1152),    # BN = 256, several tiles and a ragged tail
-    (257, 8, 128),
+    (130, 136, 640),     # two token tiles, ragged both ways
+    (200, 1000, 2048),
+    # one CTA per SM, both operands through shared memory (more than 256 tokens, fewer than 256 channels)
+    (300, 136, 640),     # BN = 128
+    (257, 8, 128),       # BN = 64
     # the two-CTA kernel
     (256, 256, 128),     # one pair tile
+    (300, 520, 1152),    # several tiles and a ragged tail
+    (100, 12296, 512),   # fewer than 256 tokens, but enough channels to fill the SM pairs
+    (200, 10240, 256),
     (600, 776, 512),     # ragged in both directions
     (300, 2560, 8192),   # two k-splits through the workspace
     (520, 2568, 8192),   # ... ragged in both directions
@@ -224,7 +228,7 @@ def test_gemm_extreme_codes(gu):
 @pytest.mark.parametrize("M,N,K", [(64, 256, 128), (3, 1024, 4096), (200, 264, 512), (130, 520, 4096),
                                    (300, 520, 640), (1024, 768, 4096), (16, 1000, 2048), (128, 520, 1024),
                                    (100, 256, 16384), (4, 1000, 14336), (1, 4096, 4096), (6, 1024, 4096), (16, 520, 14336),
-                                   (30, 8200, 1024), (64, 520, 4096), (64, 8200, 4096),
+                                   (30, 8200, 1024), (64, 520, 4096), (64, 8200, 4096), (96, 12288, 1024), (160, 520, 2048),
                                    (12, 4104, 2048), (32, 1024, 4096), (300, 2568, 8192)])
 def test_linear_output_matches_oracle_on_gpu_codes(gu, M, N, K):
     rng = np.random.default_rng(M + N + K)
