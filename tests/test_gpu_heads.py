@@ -133,6 +133,28 @@ def test_head_quantizer_edge_rows_and_row_stride(gu):
     assert np.array_equal(q2.cpu().numpy(), q) and np.array_equal(s2.cpu().numpy(), step)
 
 
+def test_head_codes_at_full_size_on_sampled_rows(gu):
+    """8192 tokens of 32 heads x 128, the launch the sweep times (a grid of 2 CTAs per SM, every
+    row group taking several rows): whole rows sampled across the range against the oracle, and
+    properties that hold for every row."""
+    n_heads, head_dim, M = 32, 128, 8192
+    K = n_heads * head_dim
+    X = _attn_out(2024, M, K)
+    q, step = _gpu_quant(gu, X, n_heads, None, 0.9)
+    assert np.all(np.isfinite(step)) and np.all(step > 0)
+    rng = np.random.default_rng(11)
+    rows = np.unique(np.concatenate([[0, 1, 3, 4, 295, 296, 1183, 1184, 1185, M - 2, M - 1],
+                                     np.arange(0, M, 13)[:8], rng.integers(0, M, 48)]))
+    q_ref, step_ref, _ = orc.quant_act_heads(X[rows], None, n_heads, 0.9)
+    assert np.abs(step[rows] / step_ref - 1).max() <= TOL_SCALE
+    frac, worst = gu.code_mismatch(q[rows], q_ref)
+    assert worst <= 1 and frac <= TOL_CODES
+    codes = orc.unpack_codes(q[::61])
+    assert codes.min() >= -8 and codes.max() <= 7
+    # the largest magnitude of a row lands on +7 or -8 (clip 0.9 puts it at 7.78 steps)
+    assert np.all(np.abs(codes.astype(np.int16)).max(axis=1) >= 7)
+
+
 def test_head_transform_then_per_head_factor_is_the_full_rotation(gu):
     """The two factors of the rotation, one on the GPU and one from the oracle, against the full
     rotation on the GPU: (I (x) H_dh)(H_h (x) I) = H_{h dh}."""
