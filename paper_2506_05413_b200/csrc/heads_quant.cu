@@ -49,19 +49,24 @@ __device__ __forceinline__ void group_sync(int id, int threads) {
 
 // kQuant: codes + step sizes; otherwise the rotated row as fp32 (test export).
 // kLowClamp: the general two-sided clamp, needed when the row maximum can reach 8.5 steps or more.
-template <int NH, bool kQuant, bool kHasPre, bool kLowClamp>
+// HD (head_dim) is a template parameter so that the strides between heads are immediates; the
+// diagonal and the clamp are uniform run-time branches.
+template <int NH, int HD, bool kQuant>
 __global__ void __launch_bounds__(kHeadsThreads, NH <= 32 ? 2 : 1)
-heads_kernel(const __half* __restrict__ x, int64_t ld, int rows, int head_dim, const float* __restrict__ pre,
+heads_kernel(const __half* __restrict__ x, int64_t ld, int rows, const float* __restrict__ pre, bool low_clamp,
              float inv_sqrt_heads, float clip, uint8_t* __restrict__ q_out, float* __restrict__ step_out,
              float* __restrict__ y_out) {
   __shared__ float red[kHeadsThreads / 32];
-  const int group_threads = head_dim >> 1;                 // threads per row: 32, 64 or 128
-  const int groups = kHeadsThreads / group_threads;
+  constexpr int head_dim = HD;
+  constexpr int group_threads = head_dim >> 1;             // threads per row: 32, 64 or 128
+  constexpr int groups = kHeadsThreads / group_threads;
+  const bool kHasPre = pre != nullptr;
+  const bool kLowClamp = low_clamp;
   const int group = threadIdx.x / group_threads;
   const int t = threadIdx.x - group * group_threads;       // this thread owns positions 2t, 2t + 1 of every head
-  const int warps = group_threads >> 5;
+  constexpr int warps = group_threads >> 5;
   const int row_stride = gridDim.x * groups;
-  const int K = NH * head_dim;
+  constexpr int K = NH * head_dim;
 
   uint32_t raw[NH];
   int m = blockIdx.x * groups + group;
@@ -184,15 +189,18 @@ int launch_heads(const void* X, int64_t rows, int64_t n_heads, int64_t head_dim,
   const int64_t cap = int64_t(device_sm_count()) * ctas_per_sm;
   if (grid > cap) grid = cap;
   auto launch = [&](auto kern) {
-    kern<<<unsigned(grid), kHeadsThreads, 0, stream>>>(static_cast<const __half*>(X), ld, int(rows), int(head_dim), pre,
-                                                      rs, clip, q_out, step_out, y_out);
+    kern<<<unsigned(grid), kHeadsThreads, 0, stream>>>(static_cast<const __half*>(X), ld, int(rows), pre, low, rs, clip,
+                                                      q_out, step_out, y_out);
     count_launch();
     return launch_status();
   };
   auto pick = [&](auto nh_tag) {
     constexpr int NH = decltype(nh_tag)::value;
-    if (pre) return low ? launch(heads_kernel<NH, kQuant, true, true>) : launch(heads_kernel<NH, kQuant, true, false>);
-    return low ? launch(heads_kernel<NH, kQuant, false, true>) : launch(heads_kernel<NH, kQuant, false, false>);
+    switch (int(head_dim)) {
+      case 64: return launch(heads_kernel<NH, 64, kQuant>);
+      case 128: return launch(heads_kernel<NH, 128, kQuant>);
+      default: return launch(heads_kernel<NH, 256, kQuant>);
+    }
   };
   switch (int(n_heads)) {
     case 8: return pick(std::integral_constant<int, 8>{});
