@@ -37,6 +37,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "decode.cuh"
 
 // defined with the row transform kernels: their timeout word
 extern "C" int smoothrot_rotate_status_word(int* value, int clear);
@@ -1289,32 +1290,6 @@ splitk_reduce_kernel(const int32_t* __restrict__ part, int splits, int M, int N,
 // not care about the order of its terms).  Sums are int32 (256 * acc), added over the warps in
 // shared memory in a fixed order: exact, and identical from run to run.
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ void mma_s8_16x8x32(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                               uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-// Volatile so that every load of a batch is issued before the first MMA that follows it in the source.
-__device__ __forceinline__ uint4 load_stream_16(const uint8_t* p) {
-  uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p));
-  return v;
-}
-__device__ __forceinline__ uint4 load_keep_16(const uint8_t* p) {
-  uint4 v;
-  asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-  return v;
-}
-
-__device__ __forceinline__ uint32_t even_codes_x16(uint32_t w) { return (w << 4) & 0xF0F0F0F0u; }
-__device__ __forceinline__ uint32_t odd_codes_x16(uint32_t w) { return w & 0xF0F0F0F0u; }
-__device__ __forceinline__ uint32_t word_of(const uint4& v, int i) { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
-
 // NT: token tiles of 8 (M <= 8 * NT); RG: row groups of 16 per CTA; U: chunks per batch and warp (two
 // batches are in flight); WARPS: warps per CTA, which split K between them.
 template <int NT, int RG, int U>

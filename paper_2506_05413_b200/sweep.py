@@ -7,7 +7,8 @@ For every shape (q/o 4096->4096, k/v 4096->1024, gate/up 4096->14336, down 14336
 every M in {1, 4, 16, 128, 512, 2048, 8192} it times the two online calls of the layer,
 smoothrot_quant_act and smoothrot_linear, on seeded synthetic activations (random-init
 weights, quantized once by smoothrot_fuse_weights), and prints time, TOP/s and GB/s; for the q/o
-shape also smoothrot_quant_act_heads (32 heads of 128), the transform the o-projection's input takes.
+shape also smoothrot_quant_act_heads (32 heads of 128), the transform the o-projection's input takes,
+and for M <= 4 with K = 4096 smoothrot_linear_decode, which does both calls in one kernel.
 
 Timing: each call is recorded into a CUDA graph per buffer set and replayed back to back
 between two CUDA events; the buffer sets rotate so that their total size exceeds twice the
@@ -76,8 +77,14 @@ def run(reps: int = 30, shapes=None, tokens=None):
                 sr.linear(xq, dx, wq, dw, Y, ws)
                 sets.append((X, xq, dx, wq, dw, Y, ws))
             torch.cuda.synchronize()
-            gq, gl, gh = [], [], []
+            gq, gl, gh, gf = [], [], [], []
             for X, xq, dx, wq, dw, Y, ws in sets:
+                if M <= 4 and K == 4096:    # both calls of the layer in one kernel
+                    sr.linear_decode(X, pre_x, case.clip_a, wq, dw, Y)
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g):
+                        sr.linear_decode(X, pre_x, case.clip_a, wq, dw, Y)
+                    gf.append(g)
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g):
                     sr.quant_act(X, pre_x, case.clip_a, xq, dx)
@@ -94,6 +101,7 @@ def run(reps: int = 30, shapes=None, tokens=None):
                 gl.append(g)
             tl = _time_graphs(torch, gl, reps)
             th = _time_graphs(torch, gh, reps) if gh else None
+            tf = _time_graphs(torch, gf, reps) if gf else None
             tq = _time_graphs(torch, gq, reps)
             assert sr.device_status() == 0
             ops = 2.0 * M * N * K
@@ -105,6 +113,8 @@ def run(reps: int = 30, shapes=None, tokens=None):
                 "weight_stream_GBs": 0.5 * N * K / tl / 1e9,
                 "buffer_sets": n_sets,
             })
+            if tf is not None:
+                rows[-1]["fused_layer_us"] = tf * 1e6
             if th is not None:
                 rows[-1]["quant_act_heads_us"] = th * 1e6
                 rows[-1]["quant_act_heads_GBs"] = (2.5 * M * K + 4 * M) / th / 1e9
@@ -169,10 +179,12 @@ def main():
             print(json.dumps(r))
         return
     print(f"{'shape':8s} {'M':>5s} {'quant us':>9s} {'GB/s':>7s} {'linear us':>10s} {'TOP/s':>8s} {'W GB/s':>8s}"
-          f" {'heads us':>9s} {'GB/s':>7s}")
+          f" {'heads us':>9s} {'GB/s':>7s} {'fused us':>9s}")
     for r in rows:
         heads = (f" {r['quant_act_heads_us']:9.1f} {r['quant_act_heads_GBs']:7.0f}"
-                 if "quant_act_heads_us" in r else "")
+                 if "quant_act_heads_us" in r else " " * 18)
+        if "fused_layer_us" in r:
+            heads += f" {r['fused_layer_us']:9.1f}"
         print(f"{r['shape']:8s} {r['M']:5d} {r['quant_act_us']:9.1f} {r['quant_act_GBs']:7.0f} "
               f"{r['linear_us']:10.1f} {r['linear_TOPS']:8.1f} {r['weight_stream_GBs']:8.0f}{heads}")
 
