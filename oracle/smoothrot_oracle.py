@@ -23,6 +23,9 @@ What follows the paper, by passage:
   quantization, group size 128 and clip ratio 0.95 (kv_quantize).
 * Fig. 2 (the feed-forward block): the down-projection input is the gated
   product sigma(gate) (.) up; quant_act_glu takes that edge in one step.
+* Section "Methodology", last paragraph: "online quantization operations are
+  integrated into the forward pass for [...] activations": the layers without
+  an online Hadamard transform quantize their input as it is (quant_act_plain).
 * Section "Methodology", "two additional Hadamard transformations integrated
   into the forward pass, as described in [QuaRot]": the paper details the one
   in front of the down-projection only.  The other sits in front of the
@@ -389,6 +392,21 @@ def quant_act(X: np.ndarray, pre_x, K: int, clip_a: float = 0.9):
     xr = rotate(X, pre_x, K).astype(np.float32)
     codes, step = quantize_rows(xr, clip_a)
     return pack_codes(codes), step, xr
+
+
+def quant_act_plain(X: np.ndarray, pre_x, clip_a: float = 0.9):
+    """The online activation quantizer of the layers that need no online Hadamard transform (the
+    paper integrates only two of those into the forward pass, in front of the down-projection and
+    of the attention output projection; every other linear layer sees activations that are already
+    in the rotated basis and only quantizes them): rows times pre_x (or one), rounded once to
+    float32, then Eq. 1's per-token symmetric quantizer with the clip ratio.
+    Returns (packed [M, K/2] u8, step [M] f32, the scaled float32 rows [M, K])."""
+    v = np.asarray(X, dtype=np.float64)
+    if pre_x is not None:
+        v = v * np.asarray(pre_x, dtype=np.float64)[None, :]
+    v = v.astype(np.float32)
+    codes, step = quantize_rows(v, clip_a)
+    return pack_codes(codes), step, v
 
 
 def rotate_heads(x: np.ndarray, pre, n_heads: int) -> np.ndarray:

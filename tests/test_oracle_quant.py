@@ -182,3 +182,36 @@ def test_dequant_output_is_the_rounded_exact_product():
     assert np.all(np.abs(y.astype(np.float64) - exact) <= np.abs(exact) * 2.0 ** -11)
     big = orc.dequant_output(np.array([[917504]], np.int32), np.array([1.0], np.float32), np.array([1.0], np.float32))
     assert np.isinf(big[0, 0])                              # IEEE overflow, not saturation
+
+
+# ---------------------------------------------------------------- the quantizer without a rotation
+def test_plain_activation_quantizer_worked_example_and_relation_to_the_rotated_path():
+    # one row, maximum 7: with clip 1 the step is 1 and the codes are the rounded values themselves
+    x = np.array([[7.0, -7.0, 0.49, 0.5, 1.5, 2.5, -0.5, -3.4]], np.float16)
+    packed, step, v = orc.quant_act_plain(x, None, 1.0)
+    assert step[0] == np.float32(1.0) and v.dtype == np.float32
+    assert list(orc.unpack_codes(packed)[0]) == [7, -7, 0, 0, 2, 2, 0, -3]       # halves go to the even neighbour
+    # clip 0.9: step 0.9, the maximum lands at 7.78 steps and saturates
+    packed, step, _ = orc.quant_act_plain(x, None, 0.9)
+    assert step[0] == np.float32(np.float32(0.9) * np.float32(7.0)) / np.float32(7.0)
+    assert list(orc.unpack_codes(packed)[0][:2]) == [7, -8]
+    # the diagonal multiplies before the quantizer: doubling every channel doubles the step, same codes
+    rng = np.random.default_rng(0)
+    X = rng.standard_normal((5, 64)).astype(np.float16)
+    p1, s1, _ = orc.quant_act_plain(X, None, 0.9)
+    p2, s2, _ = orc.quant_act_plain(X, np.full(64, 2.0, np.float32), 0.9)
+    assert np.array_equal(p1, p2) and np.array_equal(s2, 2 * s1)
+    # against the rotated path: rotating first and quantizing plainly is quant_act
+    K = 128
+    X = rng.standard_normal((4, K)).astype(np.float16)
+    q_rot, s_rot, xr = orc.quant_act(X, None, K, 0.9)
+    codes, s_plain = orc.quantize_rows(xr, 0.9)
+    assert np.array_equal(orc.pack_codes(codes), q_rot) and np.array_equal(s_plain, s_rot)
+    # a zero row and a per-channel diagonal with signs
+    X = np.zeros((1, 16), np.float16)
+    packed, step, _ = orc.quant_act_plain(X, None, 0.9)
+    assert step[0] == np.float32(1.0) and not packed.any()
+    X = np.ones((1, 8), np.float16)
+    pre = np.array([1, -1, 2, -2, 3.5, -3.5, 7, -7], np.float32)
+    packed, step, _ = orc.quant_act_plain(X, pre, 1.0)
+    assert list(orc.unpack_codes(packed)[0]) == [1, -1, 2, -2, 4, -4, 7, -7]     # 3.5 -> 4 (even), -3.5 -> -4
