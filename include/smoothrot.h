@@ -136,6 +136,20 @@ int smoothrot_quant_act(const void* X_f16, int64_t M, int64_t K, int64_t ldx,
                         uint8_t* Xq_out, float* dx_out, void* stream);
 
 /*
+ * Online activation quantizer of the layers that have no online Hadamard transform.  Methodology
+ * section, last paragraph: online quantization is integrated into the forward pass for the
+ * activations, while only two Hadamard transforms are (smoothrot_quant_act and
+ * smoothrot_quant_act_heads); every other quantized layer receives activations that are already
+ * in the rotated basis.  For every token m:
+ *     x^   = X[m][:] * pre                       (pre [K] fp32, or NULL for none)
+ *     dx[m], codes: from x^ exactly as in smoothrot_quant_act.
+ * X [M x ldx] fp16, Xq_out [M x K/2] bytes, dx_out [M] fp32.  K a multiple of 8, K <= 16384.
+ */
+int smoothrot_quant_act_plain(const void* X_f16, int64_t M, int64_t K, int64_t ldx,
+                              const float* pre, float clip_a,
+                              uint8_t* Xq_out, float* dx_out, void* stream);
+
+/*
  * Online activation path in front of the attention output projection.  Methodology section: "two
  * additional Hadamard transformations integrated into the forward pass, as described in [QuaRot]";
  * the paper spells out only the one before the down-projection (smoothrot_quant_act).  The other

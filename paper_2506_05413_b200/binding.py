@@ -28,6 +28,7 @@ SIGNATURES = {
     "smoothrot_quant_act": (_int, [_vp, _i64, _i64, _i64, _vp, _f32, _vp, _vp, _vp]),
     "smoothrot_quant_act_glu": (_int, [_vp, _vp, _i64, _i64, _i64, _i64, _vp, _f32, _vp, _vp, _vp]),
     "smoothrot_quant_act_heads": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _f32, _vp, _vp, _vp]),
+    "smoothrot_quant_act_plain": (_int, [_vp, _i64, _i64, _i64, _vp, _f32, _vp, _vp, _vp]),
     "smoothrot_kv_quant": (_int, [_vp, _i64, _i64, _i64, _f32, _vp, _vp, _vp, _vp]),
     "smoothrot_kv_dequant": (_int, [_vp, _vp, _vp, _i64, _i64, _vp, _i64, _vp]),
     "smoothrot_linear": (_int, [_vp, _vp, _i64, _vp, _vp, _i64, _i64, _vp, _i64, _vp, _sz, _vp]),
@@ -179,6 +180,11 @@ def quant_act_glu(gate, up, pre, clip_a, Xq_out, dx_out):
     _check(load().smoothrot_quant_act_glu(gp, up_p, R, K, ldg, ldu, _vec(pre, K, "pre"), float(clip_a),
                                           _ptr(Xq_out, torch.uint8, "Xq_out"), _vec(dx_out, R, "dx_out"),
                                           _stream()))
+
+
+def quant_act_plain(X, pre, clip_a, Xq_out, dx_out):
+    """smoothrot_quant_act_plain: X [M, K] fp16, no rotation -> Xq_out [M, K/2] u8, dx_out [M] f32."""
+    _quantize(load().smoothrot_quant_act_plain, X, pre, clip_a, Xq_out, dx_out, ("X", "Xq_out", "dx_out"))
 
 
 def quant_act_heads(X, n_heads, pre, clip_a, Xq_out, dx_out):

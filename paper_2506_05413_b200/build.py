@@ -17,7 +17,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 BUILD = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libsmoothrot.so")
-SOURCES = ("rotate_quant.cu", "calibrate.cu", "w4a4_gemm.cu", "clip_search.cu", "kv_quant.cu", "heads_quant.cu", "decode_fused.cu")
+SOURCES = ("rotate_quant.cu", "calibrate.cu", "w4a4_gemm.cu", "clip_search.cu", "kv_quant.cu", "heads_quant.cu", "decode_fused.cu", "plain_quant.cu")
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I" + os.path.join(ROOT, "include"), "-I" + CSRC]
 

@@ -77,8 +77,13 @@ def run(reps: int = 30, shapes=None, tokens=None):
                 sr.linear(xq, dx, wq, dw, Y, ws)
                 sets.append((X, xq, dx, wq, dw, Y, ws))
             torch.cuda.synchronize()
-            gq, gl, gh, gf = [], [], [], []
+            gq, gl, gh, gf, gp = [], [], [], [], []
             for X, xq, dx, wq, dw, Y, ws in sets:
+                sr.quant_act_plain(X, pre_x, case.clip_a, xq, dx)       # the quantizer without a rotation
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    sr.quant_act_plain(X, pre_x, case.clip_a, xq, dx)
+                gp.append(g)
                 if M <= 4 and K == 4096:    # both calls of the layer in one kernel
                     sr.linear_decode(X, pre_x, case.clip_a, wq, dw, Y)
                     g = torch.cuda.CUDAGraph()
@@ -102,6 +107,7 @@ def run(reps: int = 30, shapes=None, tokens=None):
             tl = _time_graphs(torch, gl, reps)
             th = _time_graphs(torch, gh, reps) if gh else None
             tf = _time_graphs(torch, gf, reps) if gf else None
+            tp = _time_graphs(torch, gp, reps)
             tq = _time_graphs(torch, gq, reps)
             assert sr.device_status() == 0
             ops = 2.0 * M * N * K
@@ -113,6 +119,8 @@ def run(reps: int = 30, shapes=None, tokens=None):
                 "weight_stream_GBs": 0.5 * N * K / tl / 1e9,
                 "buffer_sets": n_sets,
             })
+            rows[-1]["quant_act_plain_us"] = tp * 1e6
+            rows[-1]["quant_act_plain_GBs"] = (2.5 * M * K + 4 * M + 4 * K) / tp / 1e9
             if tf is not None:
                 rows[-1]["fused_layer_us"] = tf * 1e6
             if th is not None:
@@ -178,7 +186,7 @@ def main():
         for r in rows:
             print(json.dumps(r))
         return
-    print(f"{'shape':8s} {'M':>5s} {'quant us':>9s} {'GB/s':>7s} {'linear us':>10s} {'TOP/s':>8s} {'W GB/s':>8s}"
+    print(f"{'shape':8s} {'M':>5s} {'quant us':>9s} {'GB/s':>7s} {'plain us':>9s} {'GB/s':>7s} {'linear us':>10s} {'TOP/s':>8s} {'W GB/s':>8s}"
           f" {'heads us':>9s} {'GB/s':>7s} {'fused us':>9s}")
     for r in rows:
         heads = (f" {r['quant_act_heads_us']:9.1f} {r['quant_act_heads_GBs']:7.0f}"
@@ -186,6 +194,7 @@ def main():
         if "fused_layer_us" in r:
             heads += f" {r['fused_layer_us']:9.1f}"
         print(f"{r['shape']:8s} {r['M']:5d} {r['quant_act_us']:9.1f} {r['quant_act_GBs']:7.0f} "
+              f"{r['quant_act_plain_us']:9.1f} {r['quant_act_plain_GBs']:7.0f} "
               f"{r['linear_us']:10.1f} {r['linear_TOPS']:8.1f} {r['weight_stream_GBs']:8.0f}{heads}")
 
 

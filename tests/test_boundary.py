@@ -56,6 +56,12 @@ def test_host_side_rejections(lib):
     assert q(dummy, 4, 128, 128, None, 1.5, dummy, dummy, None) == -1
     assert q(dummy, 0, 128, 128, None, 0.9, None, None, None) == 0           # empty input is fine
     assert lib.smoothrot_fuse_weights(dummy, 4, 96, 96, None, 1.0, dummy, dummy, None) == -2
+    qp = lib.smoothrot_quant_act_plain
+    assert qp(dummy, 4, 100, 104, None, 0.9, dummy, dummy, None) == -2           # K % 8
+    assert qp(dummy, 4, 32768, 32768, None, 0.9, dummy, dummy, None) == -2       # K too long
+    assert qp(dummy, 4, 128, 64, None, 0.9, dummy, dummy, None) == -1            # ldx < K
+    assert qp(odd, 4, 128, 128, None, 0.9, dummy, dummy, None) == -3
+    assert qp(dummy, 0, 128, 128, None, 0.9, None, None, None) == 0
     qh = lib.smoothrot_quant_act_heads
     assert qh(dummy, 4, 12, 128, 1536, None, 0.9, dummy, dummy, None) == -2      # 12 heads: not a power of two
     assert qh(dummy, 4, 32, 96, 3072, None, 0.9, dummy, dummy, None) == -2       # head_dim 96
