@@ -6,7 +6,7 @@
 // are already in the rotated basis and only quantize them; this is that kernel.
 //
 // Pure streaming work, 2 bytes in and half a byte out per value: T threads share a row, a thread
-// holds up to 8 chunks of 8 consecutive values (16-byte loads, chunk c of thread t is chunk t + c T
+// holds up to 4 (long rows: 8) chunks of 8 consecutive values (16-byte loads, chunk c of thread t is chunk t + c T
 // of the row), so that the 8 codes of a chunk are exactly one aligned 32-bit word of the output and
 // no transposition is needed.  The next row's loads are in flight during the arithmetic; the threads
 // of a row meet once, for the row maximum.
@@ -17,14 +17,16 @@ namespace smoothrot {
 namespace {
 
 constexpr int kPlainThreads = 256;
-constexpr int kPlainChunks = 8;             // chunks per thread: a row has at most 8 * 8 * T values
+constexpr int kPlainMaxChunks = 8;          // chunks per thread: a row has at most 8 * 8 * 256 values
 
 __device__ __forceinline__ void plain_group_sync(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
-template <int T>                            // threads per row: 64, 128 or 256
-__global__ void __launch_bounds__(kPlainThreads, 2)
+// T: threads per row (64, 128 or 256); CH: chunks per thread (4 keeps the registers low enough for
+// four CTAs per SM, 8 is for the longest rows)
+template <int T, int CH>
+__global__ void __launch_bounds__(kPlainThreads, CH <= 4 ? 4 : 2)
 plain_quant_kernel(const __half* __restrict__ x, int64_t ld, int rows, int K, const float* __restrict__ pre,
                    bool low_clamp, float clip, uint8_t* __restrict__ q_out, float* __restrict__ step_out) {
   __shared__ float red[kPlainThreads / 32];
@@ -35,18 +37,18 @@ plain_quant_kernel(const __half* __restrict__ x, int64_t ld, int rows, int K, co
   const int chunks = K >> 3;
   const int row_stride = gridDim.x * groups;
 
-  uint4 raw[kPlainChunks];
+  uint4 raw[CH];
   int m = blockIdx.x * groups + group;
   if (m < rows) {
     const uint4* src = reinterpret_cast<const uint4*>(x + int64_t(m) * ld);
 #pragma unroll
-    for (int c = 0; c < kPlainChunks; ++c)
+    for (int c = 0; c < CH; ++c)
       raw[c] = t + c * T < chunks ? __ldcs(src + t + c * T) : make_uint4(0u, 0u, 0u, 0u);
   }
   for (; m < rows; m += row_stride) {
-    f32x2 v[kPlainChunks][4];
+    f32x2 v[CH][4];
 #pragma unroll
-    for (int c = 0; c < kPlainChunks; ++c) {
+    for (int c = 0; c < CH; ++c) {
       v[c][0] = half2_to_f32x2(raw[c].x);
       v[c][1] = half2_to_f32x2(raw[c].y);
       v[c][2] = half2_to_f32x2(raw[c].z);
@@ -56,13 +58,13 @@ plain_quant_kernel(const __half* __restrict__ x, int64_t ld, int rows, int K, co
     if (next < rows) {                       // the next row of this group is on its way during the arithmetic
       const uint4* src = reinterpret_cast<const uint4*>(x + int64_t(next) * ld);
 #pragma unroll
-      for (int c = 0; c < kPlainChunks; ++c)
+      for (int c = 0; c < CH; ++c)
         raw[c] = t + c * T < chunks ? __ldcs(src + t + c * T) : make_uint4(0u, 0u, 0u, 0u);
     }
     if (pre != nullptr) {
       const float4* p = reinterpret_cast<const float4*>(pre);
 #pragma unroll
-      for (int c = 0; c < kPlainChunks; ++c) {
+      for (int c = 0; c < CH; ++c) {
         if (t + c * T < chunks) {
           const float4 a = __ldg(p + 2 * (t + c * T)), b = __ldg(p + 2 * (t + c * T) + 1);
           v[c][0] = mul2(v[c][0], pack2(a.x, a.y));
@@ -74,7 +76,7 @@ plain_quant_kernel(const __half* __restrict__ x, int64_t ld, int rows, int K, co
     }
     float amax = 0.0f;
 #pragma unroll
-    for (int c = 0; c < kPlainChunks; ++c)
+    for (int c = 0; c < CH; ++c)
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         float a, b;
@@ -106,7 +108,7 @@ plain_quant_kernel(const __half* __restrict__ x, int64_t ld, int rows, int K, co
     const f32x2 magic2 = pack2(kMagic, kMagic);
     uint32_t* q_row = reinterpret_cast<uint32_t*>(q_out + int64_t(m) * (K >> 1));
 #pragma unroll
-    for (int c = 0; c < kPlainChunks; ++c) {
+    for (int c = 0; c < CH; ++c) {
       uint32_t lo[4], hi[4];                 // even / odd positions of the chunk
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
@@ -144,17 +146,20 @@ int smoothrot_quant_act_plain(const void* X_f16, int64_t M, int64_t K, int64_t l
   using namespace smoothrot;
   if (M < 0 || K <= 0) return SMOOTHROT_INVALID_ARG;
   if (!(clip_a > 0.0f) || clip_a > 1.0f) return SMOOTHROT_INVALID_ARG;
-  if (K % 8 != 0 || K > 8 * kPlainChunks * 256) return SMOOTHROT_UNSUPPORTED_K;
+  if (K % 8 != 0 || K > 8 * kPlainMaxChunks * 256) return SMOOTHROT_UNSUPPORTED_K;
   if (M == 0) return SMOOTHROT_OK;
   if (X_f16 == nullptr || Xq_out == nullptr || dx_out == nullptr || ldx < K || M > 0x7fffffffLL)
     return SMOOTHROT_INVALID_ARG;
   if (!aligned16(X_f16) || ldx % 8 != 0 || !aligned16(Xq_out) || (pre != nullptr && !aligned16(pre)))
     return SMOOTHROT_BAD_ALIGNMENT;
   const bool low = 7.0f / clip_a >= 8.49f;               // codes below -8 can only come up then
-  const int T = K <= 8 * kPlainChunks * 64 ? 64 : (K <= 8 * kPlainChunks * 128 ? 128 : 256);
+  // the fewest values per thread that still cover the row with at most 256 threads
+  const int64_t chunks = K / 8;
+  const int CH = chunks <= 4 * 256 ? 4 : 8;
+  const int T = chunks <= CH * 64 ? 64 : (chunks <= CH * 128 ? 128 : 256);
   const int groups = kPlainThreads / T;
   int64_t grid = (M + groups - 1) / groups;
-  const int64_t cap = int64_t(device_sm_count()) * 2;
+  const int64_t cap = int64_t(device_sm_count()) * (CH <= 4 ? 4 : 2);
   if (grid > cap) grid = cap;
   auto launch = [&](auto kern) {
     kern<<<unsigned(grid), kPlainThreads, 0, static_cast<cudaStream_t>(stream)>>>(
@@ -162,9 +167,12 @@ int smoothrot_quant_act_plain(const void* X_f16, int64_t M, int64_t K, int64_t l
     count_launch();
     return launch_status();
   };
-  if (T == 64) return launch(plain_quant_kernel<64>);
-  if (T == 128) return launch(plain_quant_kernel<128>);
-  return launch(plain_quant_kernel<256>);
+  if (CH == 4) {
+    if (T == 64) return launch(plain_quant_kernel<64, 4>);
+    if (T == 128) return launch(plain_quant_kernel<128, 4>);
+    return launch(plain_quant_kernel<256, 4>);
+  }
+  return launch(plain_quant_kernel<256, 8>);
 }
 
 }  // extern "C"
