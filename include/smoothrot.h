@@ -254,19 +254,23 @@ int smoothrot_kv_dequant(const uint8_t* q, const float* step, const float* zero,
                          int64_t C, void* Y_f16, int64_t ldy, void* stream);
 
 /*
- * The whole online layer for a handful of tokens in one kernel: smoothrot_quant_act followed by
- * smoothrot_linear (Fig. 2: "hadamard" -> "quantize" -> the quantized projection; Eq. 2 on Eq. 1's
- * integer codes), for decode steps, where two launches cost more than the work.  Every CTA rotates
- * and quantizes the tokens for itself while its share of the weights is in flight; the tokens'
- * codes and steps are the ones smoothrot_quant_act defines (same formulas, fp32 butterflies in a
- * different order of additions) and are written to Xq_out [M x K/2] / dx_out [M] when those are
- * non-NULL (device, optional).  X [M x ldx] fp16, pre [K] or NULL, Wq [N x K/2] and dw [N] from
- * smoothrot_fuse_weights, Y [M x ldy] fp16.  Supported: M <= 4 and K = 4096 (else
- * SMOOTHROT_INVALID_ARG / SMOOTHROT_UNSUPPORTED_K), N a multiple of 8.  No workspace.
+ * The whole online layer for a handful of tokens in one kernel: the online activation path
+ * followed by smoothrot_linear (Fig. 2: ["hadamard" ->] "quantize" -> the quantized projection; Eq. 2
+ * on Eq. 1's integer codes), for decode steps, where two launches cost more than the work.  Every
+ * CTA prepares the tokens for itself while its share of the weights is in flight.
+ *   rotation = 1: the tokens go through smoothrot_quant_act's path (x * pre) H / sqrt(K), same
+ *                 formulas, fp32 butterflies in a different order of additions.  K = 4096, M <= 4.
+ *   rotation = 0: through smoothrot_quant_act_plain's path (x * pre, no rotation), same codes.
+ *                 K in {1024, 2048, 4096}, M <= 8.
+ * The codes and steps are written to Xq_out [M x K/2] / dx_out [M] when those are non-NULL (device,
+ * optional).  X [M x ldx] fp16, pre [K] or NULL, Wq [N x K/2] and dw [N] from
+ * smoothrot_fuse_weights, Y [M x ldy] fp16, N a multiple of 8.  Other shapes:
+ * SMOOTHROT_INVALID_ARG (M) / SMOOTHROT_UNSUPPORTED_K.  No workspace.
  */
-int smoothrot_linear_decode(const void* X_f16, int64_t M, int64_t K, int64_t ldx, const float* pre,
-                            float clip_a, const uint8_t* Wq, const float* dw, int64_t N,
-                            void* Y_f16, int64_t ldy, uint8_t* Xq_out, float* dx_out, void* stream);
+int smoothrot_linear_decode(const void* X_f16, int64_t M, int64_t K, int64_t ldx, int rotation,
+                            const float* pre, float clip_a, const uint8_t* Wq, const float* dw,
+                            int64_t N, void* Y_f16, int64_t ldy, uint8_t* Xq_out, float* dx_out,
+                            void* stream);
 
 /* Host. Scratch bytes smoothrot_linear / smoothrot_debug_gemm_i32 want for
  * this shape (0 for shapes that need none).  With M <= 128 a shape that reports

@@ -33,7 +33,7 @@ SIGNATURES = {
     "smoothrot_kv_dequant": (_int, [_vp, _vp, _vp, _i64, _i64, _vp, _i64, _vp]),
     "smoothrot_linear": (_int, [_vp, _vp, _i64, _vp, _vp, _i64, _i64, _vp, _i64, _vp, _sz, _vp]),
     "smoothrot_linear_static_scratch": (_int, [_vp, _vp, _i64, _vp, _vp, _i64, _i64, _vp, _i64, _vp]),
-    "smoothrot_linear_decode": (_int, [_vp, _i64, _i64, _i64, _vp, _f32, _vp, _vp, _i64, _vp, _i64, _vp, _vp, _vp]),
+    "smoothrot_linear_decode": (_int, [_vp, _i64, _i64, _i64, _int, _vp, _f32, _vp, _vp, _i64, _vp, _i64, _vp, _vp, _vp]),
     "smoothrot_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "smoothrot_debug_hadamard": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp]),
     "smoothrot_debug_hadamard_heads": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _vp, _vp]),
@@ -250,8 +250,9 @@ def linear(Xq, dx, Wq, dw, Y, workspace=None):
                                    wsp, wsb, _stream()))
 
 
-def linear_decode(X, pre, clip_a, Wq, dw, Y, Xq_out=None, dx_out=None):
-    """smoothrot_linear_decode: quant_act + linear for M <= 4 tokens of K = 4096 in one kernel.
+def linear_decode(X, pre, clip_a, Wq, dw, Y, Xq_out=None, dx_out=None, rotation=True):
+    """smoothrot_linear_decode: the online activation path and linear in one kernel, for a few tokens
+    (rotation=True: quant_act's path, K = 4096, M <= 4; rotation=False: quant_act_plain's, K <= 4096, M <= 8).
     X [M, K] fp16 -> Y [M, N] fp16; Xq_out [M, K/2] u8 and dx_out [M] f32 optionally receive the codes."""
     xp, M, K, ldx = _rows(X, torch.float16, "X")
     wp, N, Kw = _packed(Wq, "Wq")
@@ -263,7 +264,7 @@ def linear_decode(X, pre, clip_a, Wq, dw, Y, Xq_out=None, dx_out=None):
     if Xq_out is not None and (Xq_out.dtype != torch.uint8 or tuple(Xq_out.shape) != (M, K // 2)
                                or not Xq_out.is_contiguous()):
         raise ValueError(f"Xq_out must be a contiguous uint8 [{M}, {K // 2}] tensor")
-    _check(load().smoothrot_linear_decode(xp, M, K, ldx, _vec(pre, K, "pre"), float(clip_a), wp, _vec(dw, N, "dw"), N,
+    _check(load().smoothrot_linear_decode(xp, M, K, ldx, 1 if rotation else 0, _vec(pre, K, "pre"), float(clip_a), wp, _vec(dw, N, "dw"), N,
                                           yp, ldy, _ptr(Xq_out, torch.uint8, "Xq_out"), _vec(dx_out, M, "dx_out"),
                                           _stream()))
 

@@ -45,7 +45,7 @@ __device__ __forceinline__ void butterflies16(float (&v)[16]) {
   }
 }
 
-__global__ void __launch_bounds__(kFusedThreads)
+__global__ void __launch_bounds__(kFusedThreads, 2)
 fused_decode_kernel(const __half* __restrict__ X, int M, int64_t ldx, const float* __restrict__ pre, float clip,
                     bool low_clamp, const uint8_t* __restrict__ Wq, int N, const float* __restrict__ dw,
                     __half* __restrict__ Y, int64_t ldy, uint8_t* __restrict__ xq_out, float* __restrict__ dx_out) {
@@ -79,19 +79,31 @@ fused_decode_kernel(const __half* __restrict__ X, int M, int64_t ldx, const floa
   const int out_m = tid >> 4;                             // the token of the output this thread finishes (tid < 128)
 
   // 2. the tokens: rotate, quantize, leave the codes in shared memory
-  for (int m = 0; m < M; ++m) {
+  // all tokens' values are requested at once: one trip to L2 instead of one per token
+  uint4 raw_all[kFusedMaxTokens][2];
+#pragma unroll
+  for (int m = 0; m < kFusedMaxTokens; ++m) {
+    const uint4* src = reinterpret_cast<const uint4*>(X + int64_t(m < M ? m : 0) * ldx + tid * 16);
+    raw_all[m][0] = __ldg(src);
+    raw_all[m][1] = __ldg(src + 1);
+  }
+  float4 scale[4];                                     // the diagonal of this thread's 16 values, once for all tokens
+#pragma unroll
+  for (int k = 0; k < 4; ++k)
+    scale[k] = pre != nullptr ? __ldg(reinterpret_cast<const float4*>(pre + tid * 16) + k) : make_float4(1.f, 1.f, 1.f, 1.f);
+#pragma unroll
+  for (int m = 0; m < kFusedMaxTokens; ++m) {
+    if (m >= M) break;
     float v[16];
     {
-      const uint4* src = reinterpret_cast<const uint4*>(X + int64_t(m) * ldx + tid * 16);
-      const uint4 a = __ldg(src), b = __ldg(src + 1);
+      const uint4 a = raw_all[m][0], b = raw_all[m][1];
       const uint32_t raw[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
 #pragma unroll
       for (int k = 0; k < 8; ++k) unpack2(half2_to_f32x2(raw[k]), v[2 * k], v[2 * k + 1]);
       if (pre != nullptr) {
-        const float4* ps = reinterpret_cast<const float4*>(pre + tid * 16);
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-          const float4 s = __ldg(ps + k);
+          const float4 s = scale[k];
           v[4 * k] *= s.x;
           v[4 * k + 1] *= s.y;
           v[4 * k + 2] *= s.z;
@@ -201,36 +213,227 @@ fused_decode_kernel(const __half* __restrict__ X, int M, int64_t ldx, const floa
   }
 }
 
+// The same layer for inputs that need no online rotation (every quantized layer quantizes its input
+// online, only two rotate it first): x * pre, per-token INT4 with the correctly rounded quotient of
+// smoothrot_quant_act_plain, then the products.  Quantizing a token is a few dozen instructions per
+// thread, so up to 8 tokens (one token tile of the MMA) are taken.  K = 1024 * CW.
+template <int CW>
+__global__ void __launch_bounds__(kFusedThreads, 2)
+fused_plain_decode_kernel(const __half* __restrict__ X, int M, int64_t ldx, const float* __restrict__ pre, float clip,
+                          const uint8_t* __restrict__ Wq, int N, const float* __restrict__ dw,
+                          __half* __restrict__ Y, int64_t ldy, uint8_t* __restrict__ xq_out,
+                          float* __restrict__ dx_out) {
+  constexpr int K = 1024 * CW;
+  constexpr int kTokens = 8;
+  constexpr int kChunks = K / 8;                                   // chunks of 8 values = packed words of a row
+  constexpr int kPerThread = (kChunks + kFusedThreads - 1) / kFusedThreads;
+  __shared__ __align__(16) uint32_t xs[kTokens][2][kChunks];      // int8 lanes (16 * code): even / odd positions
+  __shared__ float sred[kFusedWarps];
+  __shared__ float sdx[kTokens];
+  __shared__ int red[kFusedWarps][128];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = lane >> 2, t = lane & 3;
+  const int64_t row_bytes = K / 2;
+  const int groups = (N + 15) >> 4;
+  auto load_weights = [&](uint4 (&w)[CW][2], int group) {
+    const uint8_t* r0 = Wq + int64_t(min(group * 16 + g, N - 1)) * row_bytes + t * 16;
+    const uint8_t* r1 = Wq + int64_t(min(group * 16 + 8 + g, N - 1)) * row_bytes + t * 16;
+#pragma unroll
+    for (int u = 0; u < CW; ++u) {
+      const int cc = warp + u * kFusedWarps;
+      w[u][0] = load_stream_16(r0 + cc * 64);
+      w[u][1] = load_stream_16(r1 + cc * 64);
+    }
+  };
+
+  uint4 w[CW][2], w_next[CW][2];
+  int group = blockIdx.x;
+  if (group < groups) load_weights(w, group);
+  const int out_m = tid >> 4;
+
+  // all tokens' values are requested at once: one trip to L2 instead of one per token
+  uint4 raw_all[kTokens][kPerThread];
+#pragma unroll
+  for (int m = 0; m < kTokens; ++m)
+#pragma unroll
+    for (int i = 0; i < kPerThread; ++i) {
+      const int c = tid + i * kFusedThreads;
+      raw_all[m][i] = (m < M && c < kChunks) ? __ldg(reinterpret_cast<const uint4*>(X + int64_t(m) * ldx) + c)
+                                             : make_uint4(0u, 0u, 0u, 0u);
+    }
+  // the diagonal of this thread's chunks, once for all tokens
+  f32x2 scale[kPerThread][4];
+#pragma unroll
+  for (int i = 0; i < kPerThread; ++i) {
+    const int c = tid + i * kFusedThreads;
+    float4 a = make_float4(1.f, 1.f, 1.f, 1.f), b = a;
+    if (pre != nullptr && c < kChunks) {
+      a = __ldg(reinterpret_cast<const float4*>(pre) + 2 * c);
+      b = __ldg(reinterpret_cast<const float4*>(pre) + 2 * c + 1);
+    }
+    scale[i][0] = pack2(a.x, a.y);
+    scale[i][1] = pack2(a.z, a.w);
+    scale[i][2] = pack2(b.x, b.y);
+    scale[i][3] = pack2(b.z, b.w);
+  }
+#pragma unroll
+  for (int m = 0; m < kTokens; ++m) {
+    if (m >= M) break;
+    f32x2 v[kPerThread][4];
+    float amax = 0.0f;
+#pragma unroll
+    for (int i = 0; i < kPerThread; ++i) {
+      const uint4 raw = raw_all[m][i];
+      v[i][0] = half2_to_f32x2(raw.x);
+      v[i][1] = half2_to_f32x2(raw.y);
+      v[i][2] = half2_to_f32x2(raw.z);
+      v[i][3] = half2_to_f32x2(raw.w);
+      if (pre != nullptr) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) v[i][k] = mul2(v[i][k], scale[i][k]);
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        float a, b;
+        unpack2(v[i][k], a, b);
+        amax = fmaxf(amax, fmaxf(fabsf(a), fabsf(b)));
+      }
+    }
+    amax = warp_max(amax);
+    __syncthreads();                                    // sred of the previous token has been read
+    if (lane == 0) sred[warp] = amax;
+    __syncthreads();
+    amax = sred[0];
+#pragma unroll
+    for (int k = 1; k < kFusedWarps; ++k) amax = fmaxf(amax, sred[k]);
+    const float step = step_from_absmax(amax, clip);
+    if (tid == 0) {
+      sdx[m] = step;
+      if (blockIdx.x == 0 && dx_out != nullptr) dx_out[m] = step;
+    }
+    // the correctly rounded fp32 quotient x / step (reciprocal, one residual correction), rounded half
+    // to even by the 1.5 * 2^23 constant, clamped to [-8, 7]; an int8 lane is 16 * code
+    const float inv = __frcp_rn(step);
+    const f32x2 inv2 = pack2(inv, inv), neg_step2 = pack2(-step, -step), magic2 = pack2(12582912.0f, 12582912.0f);
+#pragma unroll
+    for (int i = 0; i < kPerThread; ++i) {
+      const int c = tid + i * kFusedThreads;
+      uint32_t even[4], odd[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        f32x2 q = mul2(v[i][k], inv2);
+        q = fma2(fma2(q, neg_step2, v[i][k]), inv2, q);
+        float q0, q1;
+        unpack2(add2(q, magic2), q0, q1);
+        q0 = fmaxf(fminf(q0, 12582912.0f + 7.0f), 12582912.0f - 8.0f);
+        q1 = fmaxf(fminf(q1, 12582912.0f + 7.0f), 12582912.0f - 8.0f);
+        even[k] = __float_as_uint(q0) << 4;
+        odd[k] = __float_as_uint(q1) << 4;
+      }
+      if (c < kChunks) {
+        xs[m][0][c] = __byte_perm(__byte_perm(even[0], even[1], 0x0040), __byte_perm(even[2], even[3], 0x0040), 0x5410);
+        xs[m][1][c] = __byte_perm(__byte_perm(odd[0], odd[1], 0x0040), __byte_perm(odd[2], odd[3], 0x0040), 0x5410);
+      }
+    }
+  }
+  __syncthreads();
+  if (blockIdx.x == 0 && xq_out != nullptr) {
+    for (int idx = tid; idx < M * (K / 2); idx += kFusedThreads) {
+      const int m = idx / (K / 2), i = idx - m * (K / 2);
+      const uint8_t* even = reinterpret_cast<const uint8_t*>(&xs[m][0][0]);
+      const uint8_t* odd = reinterpret_cast<const uint8_t*>(&xs[m][1][0]);
+      xq_out[int64_t(m) * (K / 2) + i] = uint8_t((even[i] >> 4) | (odd[i] & 0xF0u));
+    }
+  }
+
+  const bool live = g < M;
+  const uint32_t* xe = &xs[live ? g : 0][0][0];
+  const uint32_t* xo = &xs[live ? g : 0][1][0];
+  for (; group < groups; group += gridDim.x) {
+    const int next = group + gridDim.x;
+    if (next < groups) load_weights(w_next, next);
+    const int out_n = group * 16 + (tid & 15);
+    const float out_dw = (tid < 128 && out_n < N) ? __ldg(dw + out_n) : 0.0f;
+    int c[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int u = 0; u < CW; ++u) {
+      const int word = ((warp + u * kFusedWarps) * 4 + t) * 4;
+      uint4 b0 = make_uint4(0u, 0u, 0u, 0u), b1 = b0;
+      if (live) {
+        b0 = *reinterpret_cast<const uint4*>(xe + word);
+        b1 = *reinterpret_cast<const uint4*>(xo + word);
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t wa = word_of(w[u][0], i), wb = word_of(w[u][1], i);
+        mma_s8_16x8x32(c, even_codes_x16(wa), even_codes_x16(wb), odd_codes_x16(wa), odd_codes_x16(wb),
+                       word_of(b0, i), word_of(b1, i));
+      }
+    }
+    red[warp][(2 * t) * 16 + g] = c[0];
+    red[warp][(2 * t + 1) * 16 + g] = c[1];
+    red[warp][(2 * t) * 16 + g + 8] = c[2];
+    red[warp][(2 * t + 1) * 16 + g + 8] = c[3];
+    __syncthreads();
+    if (tid < 128 && out_m < M && out_n < N) {
+      int sum = 0;
+#pragma unroll
+      for (int k = 0; k < kFusedWarps; ++k) sum += red[k][tid];
+      sum >>= 8;
+      Y[int64_t(out_m) * ldy + out_n] = __float2half_rn(float(sum) * (sdx[out_m] * out_dw));
+    }
+    __syncthreads();
+#pragma unroll
+    for (int u = 0; u < CW; ++u) {
+      w[u][0] = w_next[u][0];
+      w[u][1] = w_next[u][1];
+    }
+  }
+}
+
 }  // namespace
 }  // namespace gemm
 }  // namespace smoothrot
 
 extern "C" {
 
-int smoothrot_linear_decode(const void* X_f16, int64_t M, int64_t K, int64_t ldx, const float* pre, float clip_a,
-                            const uint8_t* Wq, const float* dw, int64_t N, void* Y_f16, int64_t ldy,
+int smoothrot_linear_decode(const void* X_f16, int64_t M, int64_t K, int64_t ldx, int rotation, const float* pre,
+                            float clip_a, const uint8_t* Wq, const float* dw, int64_t N, void* Y_f16, int64_t ldy,
                             uint8_t* Xq_out, float* dx_out, void* stream) {
   using namespace smoothrot;
   using namespace smoothrot::gemm;
-  if (M < 0 || N < 0 || K <= 0) return SMOOTHROT_INVALID_ARG;
+  if (M < 0 || N < 0 || K <= 0 || (rotation != 0 && rotation != 1)) return SMOOTHROT_INVALID_ARG;
   if (!(clip_a > 0.0f) || clip_a > 1.0f) return SMOOTHROT_INVALID_ARG;
-  if (K != kFusedK) return SMOOTHROT_UNSUPPORTED_K;
-  if (M > kFusedMaxTokens || N % 8 != 0 || N > 0x3fffffffLL) return SMOOTHROT_INVALID_ARG;
+  if (rotation ? K != kFusedK : (K != 1024 && K != 2048 && K != 4096)) return SMOOTHROT_UNSUPPORTED_K;
+  if (M > (rotation ? kFusedMaxTokens : 8) || N % 8 != 0 || N > 0x3fffffffLL) return SMOOTHROT_INVALID_ARG;
   if (M == 0 || N == 0) return SMOOTHROT_OK;
   if (X_f16 == nullptr || Wq == nullptr || dw == nullptr || Y_f16 == nullptr || ldx < K || ldy < N)
     return SMOOTHROT_INVALID_ARG;
   if (!aligned16(X_f16) || ldx % 8 != 0 || !aligned16(Wq) || (pre != nullptr && !aligned16(pre)))
     return SMOOTHROT_BAD_ALIGNMENT;
-  const bool low = 7.0f / clip_a >= 8.49f;               // codes below -8 can only come up then
-  // every CTA rotates the tokens once, so there are no more CTAs than fit the machine at a time
-  // (2 per SM at this register count), each taking the same number of row groups
+  // every CTA prepares the tokens once, so there are no more CTAs than fit the machine at a time
+  // (2 per SM), each taking the same number of row groups
   const int64_t groups = (N + 15) / 16;
   const int64_t slots = int64_t(device_sm_count()) * 2;
   const int64_t per_cta = (groups + slots - 1) / slots;
   const unsigned grid = unsigned((groups + per_cta - 1) / per_cta);
-  fused_decode_kernel<<<grid, kFusedThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-      static_cast<const __half*>(X_f16), int(M), ldx, pre, clip_a, low, Wq, int(N), dw, static_cast<__half*>(Y_f16), ldy,
-      Xq_out, dx_out);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const __half* x = static_cast<const __half*>(X_f16);
+  __half* y = static_cast<__half*>(Y_f16);
+  if (rotation) {
+    const bool low = 7.0f / clip_a >= 8.49f;             // codes below -8 can only come up then
+    fused_decode_kernel<<<grid, kFusedThreads, 0, st>>>(x, int(M), ldx, pre, clip_a, low, Wq, int(N), dw, y, ldy,
+                                                        Xq_out, dx_out);
+  } else if (K == 4096) {
+    fused_plain_decode_kernel<4><<<grid, kFusedThreads, 0, st>>>(x, int(M), ldx, pre, clip_a, Wq, int(N), dw, y, ldy,
+                                                                 Xq_out, dx_out);
+  } else if (K == 2048) {
+    fused_plain_decode_kernel<2><<<grid, kFusedThreads, 0, st>>>(x, int(M), ldx, pre, clip_a, Wq, int(N), dw, y, ldy,
+                                                                 Xq_out, dx_out);
+  } else {
+    fused_plain_decode_kernel<1><<<grid, kFusedThreads, 0, st>>>(x, int(M), ldx, pre, clip_a, Wq, int(N), dw, y, ldy,
+                                                                 Xq_out, dx_out);
+  }
   count_launch();
   return launch_status();
 }

@@ -70,11 +70,14 @@ def test_host_side_rejections(lib):
     assert qh(odd, 4, 32, 128, 4096, None, 0.9, dummy, dummy, None) == -3
     assert qh(dummy, 0, 32, 128, 4096, None, 0.9, None, None, None) == 0
     ld = lib.smoothrot_linear_decode
-    assert ld(dummy, 5, 4096, 4096, None, 0.9, dummy, dummy, 16, dummy, 16, None, None, None) == -1    # M > 4
-    assert ld(dummy, 2, 2048, 2048, None, 0.9, dummy, dummy, 16, dummy, 16, None, None, None) == -2    # K != 4096
-    assert ld(dummy, 2, 4096, 4096, None, 0.9, dummy, dummy, 12, dummy, 16, None, None, None) == -1    # N % 8
-    assert ld(odd, 2, 4096, 4096, None, 0.9, dummy, dummy, 16, dummy, 16, None, None, None) == -3
-    assert ld(dummy, 0, 4096, 4096, None, 0.9, dummy, dummy, 16, dummy, 16, None, None, None) == 0
+    assert ld(dummy, 5, 4096, 4096, 1, None, 0.9, dummy, dummy, 16, dummy, 16, None, None, None) == -1    # M > 4, rotated
+    assert ld(dummy, 9, 4096, 4096, 0, None, 0.9, dummy, dummy, 16, dummy, 16, None, None, None) == -1    # M > 8, plain
+    assert ld(dummy, 2, 2048, 2048, 1, None, 0.9, dummy, dummy, 16, dummy, 16, None, None, None) == -2    # rotated: K = 4096 only
+    assert ld(dummy, 2, 8192, 8192, 0, None, 0.9, dummy, dummy, 16, dummy, 16, None, None, None) == -2    # plain: K <= 4096
+    assert ld(dummy, 2, 4096, 4096, 2, None, 0.9, dummy, dummy, 16, dummy, 16, None, None, None) == -1    # rotation flag
+    assert ld(dummy, 2, 4096, 4096, 1, None, 0.9, dummy, dummy, 12, dummy, 16, None, None, None) == -1    # N % 8
+    assert ld(odd, 2, 4096, 4096, 0, None, 0.9, dummy, dummy, 16, dummy, 16, None, None, None) == -3
+    assert ld(dummy, 0, 4096, 4096, 1, None, 0.9, dummy, dummy, 16, dummy, 16, None, None, None) == 0
     lin = lib.smoothrot_linear
     assert lin(dummy, dummy, 4, dummy, dummy, 8, 100, dummy, 8, None, 0, None) == -2   # K % 128
     assert lin(dummy, dummy, 4, dummy, dummy, 12, 128, dummy, 16, None, 0, None) == -1  # N % 8

@@ -32,21 +32,22 @@ def _acts(seed, M):
                              outlier_tokens=np.arange(0, M, 2))
 
 
-def _weights(seed, N):
+def _weights(seed, N, width=K):
     rng = np.random.default_rng(seed)
-    wq = orc.pack_codes(synth.random_codes(seed, N, K))
+    wq = orc.pack_codes(synth.random_codes(seed, N, width))
     dw = rng.uniform(1e-4, 4e-3, N).astype(np.float32)
     return wq, dw
 
 
-def _run(gu, X, pre, clip, wq, dw, export=True):
+def _run(gu, X, pre, clip, wq, dw, export=True, rotation=True):
     import torch
     from paper_2506_05413_b200 import binding as sr
     M, N = X.shape[0], wq.shape[0]
     Y = torch.full((M, N), float("nan"), dtype=torch.float16, device=gu.DEV)
     xq = torch.full((M, K // 2), 0x5A, dtype=torch.uint8, device=gu.DEV) if export else None
     dx = torch.full((M,), float("nan"), dtype=torch.float32, device=gu.DEV) if export else None
-    sr.linear_decode(gu.dev(X), gu.dev(pre) if pre is not None else None, clip, gu.dev(wq), gu.dev(dw), Y, xq, dx)
+    sr.linear_decode(gu.dev(X), gu.dev(pre) if pre is not None else None, clip, gu.dev(wq), gu.dev(dw), Y, xq, dx,
+                     rotation=rotation)
     torch.cuda.synchronize()
     return (Y.cpu().numpy(), xq.cpu().numpy() if export else None, dx.cpu().numpy() if export else None)
 
@@ -104,6 +105,45 @@ def test_fused_decode_clip_ratios_and_edge_rows(gu, clip):
     # the unit vector: |x^| / step = 7 / clip everywhere, so +-7 without clipping, +7 / -8 once it saturates
     assert set(np.unique(codes[2])) <= ({7, -7} if clip == 1.0 else {7, -8})
     assert gu.rowwise_rel(Y, orc.linear(xq, dx, wq, dw)) <= TOL_OUT
+
+
+@pytest.mark.parametrize("M", [1, 3, 4, 8])
+@pytest.mark.parametrize("N,width", [(4096, 4096), (1000, 4096), (14336, 4096), (264, 2048), (72, 1024)])
+@pytest.mark.parametrize("use_pre", [False, True])
+def test_fused_decode_without_rotation(gu, M, N, width, use_pre):
+    """rotation = 0: the tokens take smoothrot_quant_act_plain's path; codes identical to the oracle's
+    (correctly rounded quotient), outputs against the oracle's layer on those codes."""
+    rng = np.random.default_rng(M + N + width)
+    ch = np.sort(rng.choice(width, size=3, replace=False))
+    X = synth.activations(rng, M, width, law="normal", outlier_channels=ch, outlier_gain=300.0,
+                          outlier_tokens=np.arange(0, M, 3))
+    X[M - 1, :] = 0 if M > 2 else X[M - 1, :]
+    pre = (rng.uniform(0.02, 8.0, width) * (rng.integers(0, 2, width) * 2 - 1)).astype(np.float32) if use_pre else None
+    wq, dw = _weights(N + M, N, width)
+    import torch
+    from paper_2506_05413_b200 import binding as sr
+    Y = torch.full((M, N), float("nan"), dtype=torch.float16, device=gu.DEV)
+    xq = torch.full((M, width // 2), 0x5A, dtype=torch.uint8, device=gu.DEV)
+    dx = torch.full((M,), float("nan"), dtype=torch.float32, device=gu.DEV)
+    sr.linear_decode(gu.dev(X), gu.dev(pre) if pre is not None else None, 0.9, gu.dev(wq), gu.dev(dw), Y, xq, dx,
+                     rotation=False)
+    torch.cuda.synchronize()
+    Y, xq, dx = Y.cpu().numpy(), xq.cpu().numpy(), dx.cpu().numpy()
+    q_ref, step_ref, _ = orc.quant_act_plain(X, pre, 0.9)
+    assert np.abs(dx / step_ref - 1).max() <= TOL_SCALE
+    frac, worst = gu.code_mismatch(xq, q_ref)
+    assert worst <= 1 and frac <= max(TOL_CODES, 1.5 / xq.size / 2)
+    assert np.isfinite(Y.astype(np.float32)).all()
+    assert gu.rowwise_rel(Y, orc.linear(xq, dx, wq, dw)) <= TOL_OUT
+    # the two-call path on the same inputs gives the same outputs bit for bit when the codes agree
+    q2 = torch.empty((M, width // 2), dtype=torch.uint8, device=gu.DEV)
+    s2 = torch.empty(M, dtype=torch.float32, device=gu.DEV)
+    Y2 = torch.empty((M, N), dtype=torch.float16, device=gu.DEV)
+    sr.quant_act_plain(gu.dev(X), gu.dev(pre) if pre is not None else None, 0.9, q2, s2)
+    sr.linear(q2, s2, gu.dev(wq), gu.dev(dw), Y2)
+    torch.cuda.synchronize()
+    assert np.array_equal(q2.cpu().numpy(), xq) and np.array_equal(s2.cpu().numpy(), dx)
+    assert np.array_equal(Y2.cpu().numpy(), Y)
 
 
 def test_fused_decode_rejects_what_it_does_not_cover(gu):

@@ -80,3 +80,26 @@ def test_static_scratch_entry_point_refuses_oversized_shapes_and_needs_no_scratc
     sr.linear_static_scratch(xq, dx, wq, dw, Y1)
     torch.cuda.synchronize()
     assert torch.equal(Y0, Y1)
+
+
+def test_static_scratch_entry_point_on_prefill_shapes_whose_k_split_is_optional():
+    """M >= 256 with few tiles and a long K: smoothrot_linear splits K through the workspace.  The
+    no-allocation entry point does the same inside its array when the partial sums fit, and runs
+    unsplit when they do not; either way the outputs equal smoothrot_linear's bit for bit."""
+    import torch
+    from paper_2506_05413_b200 import build, binding as sr
+    build.build()
+    dev = "cuda:0"
+    t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+    for call, (M, N, K, fits) in enumerate([(300, 2568, 8192, True), (512, 4096, 8192, False)]):
+        need = sr.workspace_bytes(M, N, K)
+        assert need > 0 and (need <= sr.STATIC_SCRATCH_BYTES) == fits
+        xq, dx, wq, dw = (t(a) for a in _case(300 + call, M, N, K))
+        ws = torch.empty(need, dtype=torch.uint8, device=dev)
+        Y_ref = torch.empty((M, N), dtype=torch.float16, device=dev)
+        sr.linear(xq, dx, wq, dw, Y_ref, ws)
+        Y = torch.full((M, N), float("nan"), dtype=torch.float16, device=dev)
+        sr.linear_static_scratch(xq, dx, wq, dw, Y)
+        torch.cuda.synchronize()
+        assert sr.device_status() == 0
+        assert torch.equal(Y, Y_ref)
