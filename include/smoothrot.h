@@ -272,6 +272,14 @@ int smoothrot_linear_decode(const void* X_f16, int64_t M, int64_t K, int64_t ldx
                             int64_t N, void* Y_f16, int64_t ldy, uint8_t* Xq_out, float* dx_out,
                             void* stream);
 
+/* As smoothrot_linear_decode, for the attention output projection: the tokens go through
+ * smoothrot_quant_act_heads' path, (x * pre)(H_heads (x) I_head_dim) / sqrt(heads).  Supported:
+ * 32 heads of 128 (K = 4096), M <= 4. */
+int smoothrot_linear_decode_heads(const void* X_f16, int64_t M, int64_t n_heads, int64_t head_dim,
+                                  int64_t ldx, const float* pre, float clip_a, const uint8_t* Wq,
+                                  const float* dw, int64_t N, void* Y_f16, int64_t ldy,
+                                  uint8_t* Xq_out, float* dx_out, void* stream);
+
 /* Host. Scratch bytes smoothrot_linear / smoothrot_debug_gemm_i32 want for
  * this shape (0 for shapes that need none).  With M <= 128 a shape that reports
  * a size cannot run without it (SMOOTHROT_WORKSPACE_TOO_SMALL).  With M >= 256 the

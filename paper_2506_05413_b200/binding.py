@@ -33,6 +33,7 @@ SIGNATURES = {
     "smoothrot_kv_dequant": (_int, [_vp, _vp, _vp, _i64, _i64, _vp, _i64, _vp]),
     "smoothrot_linear": (_int, [_vp, _vp, _i64, _vp, _vp, _i64, _i64, _vp, _i64, _vp, _sz, _vp]),
     "smoothrot_linear_static_scratch": (_int, [_vp, _vp, _i64, _vp, _vp, _i64, _i64, _vp, _i64, _vp]),
+    "smoothrot_linear_decode_heads": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _f32, _vp, _vp, _i64, _vp, _i64, _vp, _vp, _vp]),
     "smoothrot_linear_decode": (_int, [_vp, _i64, _i64, _i64, _int, _vp, _f32, _vp, _vp, _i64, _vp, _i64, _vp, _vp, _vp]),
     "smoothrot_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "smoothrot_debug_hadamard": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp]),
@@ -267,6 +268,24 @@ def linear_decode(X, pre, clip_a, Wq, dw, Y, Xq_out=None, dx_out=None, rotation=
     _check(load().smoothrot_linear_decode(xp, M, K, ldx, 1 if rotation else 0, _vec(pre, K, "pre"), float(clip_a), wp, _vec(dw, N, "dw"), N,
                                           yp, ldy, _ptr(Xq_out, torch.uint8, "Xq_out"), _vec(dx_out, M, "dx_out"),
                                           _stream()))
+
+
+def linear_decode_heads(X, n_heads, pre, clip_a, Wq, dw, Y, Xq_out=None, dx_out=None):
+    """smoothrot_linear_decode_heads: quant_act_heads' path and linear in one kernel (32 heads of 128, M <= 4)."""
+    xp, M, K, ldx = _rows(X, torch.float16, "X")
+    wp, N, Kw = _packed(Wq, "Wq")
+    if K != Kw or n_heads <= 0 or K % n_heads:
+        raise ValueError("X, Wq and n_heads disagree on K")
+    yp, My, Ny, ldy = _rows(Y, torch.float16, "Y")
+    if (My, Ny) != (M, N):
+        raise ValueError(f"Y must be [{M}, {N}]")
+    if Xq_out is not None and (Xq_out.dtype != torch.uint8 or tuple(Xq_out.shape) != (M, K // 2)
+                               or not Xq_out.is_contiguous()):
+        raise ValueError(f"Xq_out must be a contiguous uint8 [{M}, {K // 2}] tensor")
+    _check(load().smoothrot_linear_decode_heads(xp, M, int(n_heads), K // int(n_heads), ldx, _vec(pre, K, "pre"),
+                                                float(clip_a), wp, _vec(dw, N, "dw"), N, yp, ldy,
+                                                _ptr(Xq_out, torch.uint8, "Xq_out"), _vec(dx_out, M, "dx_out"),
+                                                _stream()))
 
 
 STATIC_SCRATCH_BYTES = 8 * 1024 * 1024   # SMOOTHROT_STATIC_SCRATCH_BYTES in the header

@@ -45,6 +45,92 @@ __device__ __forceinline__ void butterflies16(float (&v)[16]) {
   }
 }
 
+// This warp's weights for one row group of 16 output channels: CW chunks of 64 bytes of rows g and
+// g + 8 (a row past the end repeats the last one).  K = 1024 * CW.
+template <int CW>
+__device__ __forceinline__ void fused_load_weights(uint4 (&w)[CW][2], const uint8_t* __restrict__ Wq, int N, int group,
+                                                   int warp, int g, int t) {
+  constexpr int64_t row_bytes = 1024 * CW / 2;
+  const uint8_t* r0 = Wq + int64_t(min(group * 16 + g, N - 1)) * row_bytes + t * 16;
+  const uint8_t* r1 = Wq + int64_t(min(group * 16 + 8 + g, N - 1)) * row_bytes + t * 16;
+#pragma unroll
+  for (int u = 0; u < CW; ++u) {
+    const int cc = warp + u * kFusedWarps;
+    w[u][0] = load_stream_16(r0 + cc * 64);
+    w[u][1] = load_stream_16(r1 + cc * 64);
+  }
+}
+
+// The product phase shared by the fused kernels: row groups `group`, group + gridDim.x, ... against the
+// tokens' codes in shared memory (xs: per token the even-position and the odd-position plane of int8
+// lanes, K / 8 words each; tokens past M contribute zeros); rows g, g + 8 of a group against token g;
+// the next group's weights are in flight during the products.  `w` holds the first group's weights.
+template <int CW>
+__device__ __forceinline__ void fused_products(const uint32_t* xs, const float* sdx, int (*red)[128], uint4 (&w)[CW][2],
+                                               int group, int groups, const uint8_t* __restrict__ Wq, int M, int N,
+                                               const float* __restrict__ dw, __half* __restrict__ Y, int64_t ldy) {
+  constexpr int kPlane = 1024 * CW / 8;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = lane >> 2, t = lane & 3;
+  const int out_m = tid >> 4;                             // the token of the output this thread finishes (tid < 128)
+  const bool live = g < M;
+  const uint32_t* xe = xs + (live ? g : 0) * 2 * kPlane;
+  const uint32_t* xo = xe + kPlane;
+  uint4 w_next[CW][2];
+  for (; group < groups; group += gridDim.x) {
+    const int next = group + gridDim.x;
+    if (next < groups) fused_load_weights<CW>(w_next, Wq, N, next, warp, g, t);
+    const int out_n = group * 16 + (tid & 15);
+    const float out_dw = (tid < 128 && out_n < N) ? __ldg(dw + out_n) : 0.0f;
+    int c[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int u = 0; u < CW; ++u) {
+      const int word = ((warp + u * kFusedWarps) * 4 + t) * 4;   // first packed word of this lane's 16 bytes
+      uint4 b0 = make_uint4(0u, 0u, 0u, 0u), b1 = b0;
+      if (live) {
+        b0 = *reinterpret_cast<const uint4*>(xe + word);
+        b1 = *reinterpret_cast<const uint4*>(xo + word);
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t wa = word_of(w[u][0], i), wb = word_of(w[u][1], i);
+        mma_s8_16x8x32(c, even_codes_x16(wa), even_codes_x16(wb), odd_codes_x16(wa), odd_codes_x16(wb),
+                       word_of(b0, i), word_of(b1, i));
+      }
+    }
+    // add the warps' sums (int32, fixed order), dequantize, store
+    red[warp][(2 * t) * 16 + g] = c[0];
+    red[warp][(2 * t + 1) * 16 + g] = c[1];
+    red[warp][(2 * t) * 16 + g + 8] = c[2];
+    red[warp][(2 * t + 1) * 16 + g + 8] = c[3];
+    __syncthreads();
+    if (tid < 128 && out_m < M && out_n < N) {
+      int sum = 0;
+#pragma unroll
+      for (int k = 0; k < kFusedWarps; ++k) sum += red[k][tid];
+      sum >>= 8;                                         // the sums are 256 * acc, exactly
+      Y[int64_t(out_m) * ldy + out_n] = __float2half_rn(float(sum) * (sdx[out_m] * out_dw));
+    }
+    __syncthreads();                                     // red is written again by the next group
+#pragma unroll
+    for (int u = 0; u < CW; ++u) {
+      w[u][0] = w_next[u][0];
+      w[u][1] = w_next[u][1];
+    }
+  }
+}
+
+// Export of the packed codes (CTA 0 only): byte i of a row = code 2i (bits 0-3) | code 2i + 1 (bits 4-7);
+// codes 2i and 2i + 1 sit in lane i of the two planes.
+__device__ __forceinline__ void fused_export_codes(const uint32_t* xs, int M, int K, uint8_t* __restrict__ xq_out) {
+  const uint8_t* lanes = reinterpret_cast<const uint8_t*>(xs);
+  for (int idx = threadIdx.x; idx < M * (K / 2); idx += kFusedThreads) {
+    const int m = idx / (K / 2), i = idx - m * (K / 2);
+    const uint8_t even = lanes[(m * 2) * (K / 2) + i], odd = lanes[(m * 2 + 1) * (K / 2) + i];
+    xq_out[int64_t(m) * (K / 2) + i] = uint8_t((even >> 4) | (odd & 0xF0u));
+  }
+}
+
 __global__ void __launch_bounds__(kFusedThreads, 2)
 fused_decode_kernel(const __half* __restrict__ X, int M, int64_t ldx, const float* __restrict__ pre, float clip,
                     bool low_clamp, const uint8_t* __restrict__ Wq, int N, const float* __restrict__ dw,
@@ -57,26 +143,12 @@ fused_decode_kernel(const __half* __restrict__ X, int M, int64_t ldx, const floa
   __shared__ int red[kFusedWarps][128];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t = lane & 3;
-  const int64_t row_bytes = K / 2;
   const int groups = (N + 15) >> 4;                       // row groups of 16 output channels
-  // this warp's weights for one row group: 4 chunks of 64 bytes of rows g and g + 8
-  // (a row past the end repeats the last one)
-  auto load_weights = [&](uint4 (&w)[kFusedChunksPerWarp][2], int group) {
-    const uint8_t* r0 = Wq + int64_t(min(group * 16 + g, N - 1)) * row_bytes + t * 16;
-    const uint8_t* r1 = Wq + int64_t(min(group * 16 + 8 + g, N - 1)) * row_bytes + t * 16;
-#pragma unroll
-    for (int u = 0; u < kFusedChunksPerWarp; ++u) {
-      const int cc = warp + u * kFusedWarps;
-      w[u][0] = load_stream_16(r0 + cc * 64);
-      w[u][1] = load_stream_16(r1 + cc * 64);
-    }
-  };
 
   // 1. the weights of the first row group are on their way before anything else
-  uint4 w[kFusedChunksPerWarp][2], w_next[kFusedChunksPerWarp][2];
-  int group = blockIdx.x;
-  if (group < groups) load_weights(w, group);
-  const int out_m = tid >> 4;                             // the token of the output this thread finishes (tid < 128)
+  uint4 w[kFusedChunksPerWarp][2];
+  const int group = blockIdx.x;
+  if (group < groups) fused_load_weights<kFusedChunksPerWarp>(w, Wq, N, group, warp, g, t);
 
   // 2. the tokens: rotate, quantize, leave the codes in shared memory
   // all tokens' values are requested at once: one trip to L2 instead of one per token
@@ -154,63 +226,10 @@ fused_decode_kernel(const __half* __restrict__ X, int M, int64_t ldx, const floa
     // the next token's first write to sred comes after two more barriers; buf is free since the barrier above
   }
   __syncthreads();
-  if (blockIdx.x == 0 && xq_out != nullptr) {
-    // export of the packed codes: byte i of a row = code 2i (bits 0-3) | code 2i+1 (bits 4-7)
-    for (int idx = tid; idx < M * (K / 2); idx += kFusedThreads) {
-      const int m = idx / (K / 2), i = idx - m * (K / 2);
-      const uint8_t* even = reinterpret_cast<const uint8_t*>(&xs[m][0][0]);
-      const uint8_t* odd = reinterpret_cast<const uint8_t*>(&xs[m][1][0]);
-      // codes 2i and 2i + 1 sit in lane i of their planes (word i >> 2, slot i & 3)
-      xq_out[int64_t(m) * (K / 2) + i] = uint8_t((even[i] >> 4) | (odd[i] & 0xF0u));
-    }
-  }
+  if (blockIdx.x == 0 && xq_out != nullptr) fused_export_codes(&xs[0][0][0], M, K, xq_out);
 
-  // 3. row groups blockIdx.x, blockIdx.x + gridDim.x, ...: rows g, g + 8 of the group against token g
-  //    (tokens past M contribute zeros); the next group's weights are in flight during the products
-  const bool live = g < M;
-  const uint32_t* xe = &xs[live ? g : 0][0][0];
-  const uint32_t* xo = &xs[live ? g : 0][1][0];
-  for (; group < groups; group += gridDim.x) {
-    const int next = group + gridDim.x;
-    if (next < groups) load_weights(w_next, next);
-    const int out_n = group * 16 + (tid & 15);
-    const float out_dw = (tid < 128 && out_n < N) ? __ldg(dw + out_n) : 0.0f;
-    int c[4] = {0, 0, 0, 0};
-#pragma unroll
-    for (int u = 0; u < kFusedChunksPerWarp; ++u) {
-      const int word = ((warp + u * kFusedWarps) * 4 + t) * 4;   // first packed word of this lane's 16 bytes
-      uint4 b0 = make_uint4(0u, 0u, 0u, 0u), b1 = b0;
-      if (live) {
-        b0 = *reinterpret_cast<const uint4*>(xe + word);
-        b1 = *reinterpret_cast<const uint4*>(xo + word);
-      }
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const uint32_t wa = word_of(w[u][0], i), wb = word_of(w[u][1], i);
-        mma_s8_16x8x32(c, even_codes_x16(wa), even_codes_x16(wb), odd_codes_x16(wa), odd_codes_x16(wb),
-                       word_of(b0, i), word_of(b1, i));
-      }
-    }
-    // add the warps' sums (int32, fixed order), dequantize, store
-    red[warp][(2 * t) * 16 + g] = c[0];
-    red[warp][(2 * t + 1) * 16 + g] = c[1];
-    red[warp][(2 * t) * 16 + g + 8] = c[2];
-    red[warp][(2 * t + 1) * 16 + g + 8] = c[3];
-    __syncthreads();
-    if (tid < 128 && out_m < M && out_n < N) {
-      int sum = 0;
-#pragma unroll
-      for (int k = 0; k < kFusedWarps; ++k) sum += red[k][tid];
-      sum >>= 8;                                         // the sums are 256 * acc, exactly
-      Y[int64_t(out_m) * ldy + out_n] = __float2half_rn(float(sum) * (sdx[out_m] * out_dw));
-    }
-    __syncthreads();                                     // red is written again by the next group
-#pragma unroll
-    for (int u = 0; u < kFusedChunksPerWarp; ++u) {
-      w[u][0] = w_next[u][0];
-      w[u][1] = w_next[u][1];
-    }
-  }
+  // 3. the products, row group after row group
+  fused_products<kFusedChunksPerWarp>(&xs[0][0][0], sdx, red, w, group, groups, Wq, M, N, dw, Y, ldy);
 }
 
 // The same layer for inputs that need no online rotation (every quantized layer quantizes its input
@@ -233,23 +252,10 @@ fused_plain_decode_kernel(const __half* __restrict__ X, int M, int64_t ldx, cons
   __shared__ int red[kFusedWarps][128];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t = lane & 3;
-  const int64_t row_bytes = K / 2;
   const int groups = (N + 15) >> 4;
-  auto load_weights = [&](uint4 (&w)[CW][2], int group) {
-    const uint8_t* r0 = Wq + int64_t(min(group * 16 + g, N - 1)) * row_bytes + t * 16;
-    const uint8_t* r1 = Wq + int64_t(min(group * 16 + 8 + g, N - 1)) * row_bytes + t * 16;
-#pragma unroll
-    for (int u = 0; u < CW; ++u) {
-      const int cc = warp + u * kFusedWarps;
-      w[u][0] = load_stream_16(r0 + cc * 64);
-      w[u][1] = load_stream_16(r1 + cc * 64);
-    }
-  };
-
-  uint4 w[CW][2], w_next[CW][2];
-  int group = blockIdx.x;
-  if (group < groups) load_weights(w, group);
-  const int out_m = tid >> 4;
+  uint4 w[CW][2];
+  const int group = blockIdx.x;
+  if (group < groups) fused_load_weights<CW>(w, Wq, N, group, warp, g, t);
 
   // all tokens' values are requested at once: one trip to L2 instead of one per token
   uint4 raw_all[kTokens][kPerThread];
@@ -337,58 +343,94 @@ fused_plain_decode_kernel(const __half* __restrict__ X, int M, int64_t ldx, cons
     }
   }
   __syncthreads();
-  if (blockIdx.x == 0 && xq_out != nullptr) {
-    for (int idx = tid; idx < M * (K / 2); idx += kFusedThreads) {
-      const int m = idx / (K / 2), i = idx - m * (K / 2);
-      const uint8_t* even = reinterpret_cast<const uint8_t*>(&xs[m][0][0]);
-      const uint8_t* odd = reinterpret_cast<const uint8_t*>(&xs[m][1][0]);
-      xq_out[int64_t(m) * (K / 2) + i] = uint8_t((even[i] >> 4) | (odd[i] & 0xF0u));
-    }
-  }
+  if (blockIdx.x == 0 && xq_out != nullptr) fused_export_codes(&xs[0][0][0], M, K, xq_out);
+  fused_products<CW>(&xs[0][0][0], sdx, red, w, group, groups, Wq, M, N, dw, Y, ldy);
+}
 
-  const bool live = g < M;
-  const uint32_t* xe = &xs[live ? g : 0][0][0];
-  const uint32_t* xo = &xs[live ? g : 0][1][0];
-  for (; group < groups; group += gridDim.x) {
-    const int next = group + gridDim.x;
-    if (next < groups) load_weights(w_next, next);
-    const int out_n = group * 16 + (tid & 15);
-    const float out_dw = (tid < 128 && out_n < N) ? __ldg(dw + out_n) : 0.0f;
-    int c[4] = {0, 0, 0, 0};
+// The same layer for the attention output projection: the tokens go through the head-mixing
+// transform of smoothrot_quant_act_heads, (x * pre)(H_32 (x) I_128) / sqrt(32), 5 butterfly stages.
+// 64 threads rotate one token (a thread owns two neighbouring positions of every head, as in
+// heads_quant.cu), so the four groups of the CTA take up to four tokens side by side.
+__global__ void __launch_bounds__(kFusedThreads, 2)
+fused_heads_decode_kernel(const __half* __restrict__ X, int M, int64_t ldx, const float* __restrict__ pre, float clip,
+                          bool low_clamp, const uint8_t* __restrict__ Wq, int N, const float* __restrict__ dw,
+                          __half* __restrict__ Y, int64_t ldy, uint8_t* __restrict__ xq_out,
+                          float* __restrict__ dx_out) {
+  constexpr int K = kFusedK, NH = 32, HD = 128, CW = kFusedChunksPerWarp;
+  __shared__ __align__(16) uint32_t xs[kFusedMaxTokens][2][K / 8];
+  __shared__ float sred[kFusedWarps];
+  __shared__ float sdx[kFusedMaxTokens];
+  __shared__ int red[kFusedWarps][128];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = lane >> 2, t = lane & 3;
+  const int groups = (N + 15) >> 4;
+  uint4 w[CW][2];
+  const int group = blockIdx.x;
+  if (group < groups) fused_load_weights<CW>(w, Wq, N, group, warp, g, t);
+
+  const int m = tid >> 6;                 // the token this thread works on
+  const int p = tid & 63;                 // it owns positions 2p, 2p + 1 of every head
+  const bool have = m < M;
+  f32x2 v[NH];
+  {
+    const uint32_t* src = reinterpret_cast<const uint32_t*>(X + int64_t(have ? m : 0) * ldx) + p;
 #pragma unroll
-    for (int u = 0; u < CW; ++u) {
-      const int word = ((warp + u * kFusedWarps) * 4 + t) * 4;
-      uint4 b0 = make_uint4(0u, 0u, 0u, 0u), b1 = b0;
-      if (live) {
-        b0 = *reinterpret_cast<const uint4*>(xe + word);
-        b1 = *reinterpret_cast<const uint4*>(xo + word);
+    for (int h = 0; h < NH; ++h) v[h] = half2_to_f32x2(__ldg(src + h * (HD / 2)));
+    if (pre != nullptr) {
+      const float2* ps = reinterpret_cast<const float2*>(pre) + p;
+#pragma unroll
+      for (int h = 0; h < NH; ++h) {
+        const float2 sc = __ldg(ps + h * (HD / 2));
+        v[h] = mul2(v[h], pack2(sc.x, sc.y));
       }
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const uint32_t wa = word_of(w[u][0], i), wb = word_of(w[u][1], i);
-        mma_s8_16x8x32(c, even_codes_x16(wa), even_codes_x16(wb), odd_codes_x16(wa), odd_codes_x16(wb),
-                       word_of(b0, i), word_of(b1, i));
-      }
-    }
-    red[warp][(2 * t) * 16 + g] = c[0];
-    red[warp][(2 * t + 1) * 16 + g] = c[1];
-    red[warp][(2 * t) * 16 + g + 8] = c[2];
-    red[warp][(2 * t + 1) * 16 + g + 8] = c[3];
-    __syncthreads();
-    if (tid < 128 && out_m < M && out_n < N) {
-      int sum = 0;
-#pragma unroll
-      for (int k = 0; k < kFusedWarps; ++k) sum += red[k][tid];
-      sum >>= 8;
-      Y[int64_t(out_m) * ldy + out_n] = __float2half_rn(float(sum) * (sdx[out_m] * out_dw));
-    }
-    __syncthreads();
-#pragma unroll
-    for (int u = 0; u < CW; ++u) {
-      w[u][0] = w_next[u][0];
-      w[u][1] = w_next[u][1];
     }
   }
+#pragma unroll
+  for (int hb = 1; hb < NH; hb <<= 1) {
+#pragma unroll
+    for (int k = 0; k < NH; ++k) {
+      if ((k & hb) == 0) {
+        const f32x2 a = v[k], b = v[k + hb];
+        v[k] = add2(a, b);
+        v[k + hb] = sub2(a, b);
+      }
+    }
+  }
+  float amax = 0.0f;
+#pragma unroll
+  for (int h = 0; h < NH; ++h) {
+    float a, b;
+    unpack2(v[h], a, b);
+    amax = fmaxf(amax, fmaxf(fabsf(a), fabsf(b)));
+  }
+  amax = warp_max(amax);
+  if (lane == 0) sred[warp] = amax;
+  __syncthreads();
+  amax = fmaxf(sred[2 * m], sred[2 * m + 1]) * 0.17677669529663687f;    // 1 / sqrt(32): the normalised maximum
+  const float step = step_from_absmax(amax, clip);
+  if (p == 0 && have) {
+    sdx[m] = step;
+    if (blockIdx.x == 0 && dx_out != nullptr) dx_out[m] = step;
+  }
+  if (have) {
+    const float inv = __frcp_rn(step) * 0.17677669529663687f;           // 1 / step for the unnormalised values
+    uint8_t* even = reinterpret_cast<uint8_t*>(&xs[m][0][0]);
+    uint8_t* odd = reinterpret_cast<uint8_t*>(&xs[m][1][0]);
+#pragma unroll
+    for (int h = 0; h < NH; ++h) {
+      float a, b;
+      unpack2(v[h], a, b);
+      float q0 = __fmaf_rn(a, inv, 12582912.0f), q1 = __fmaf_rn(b, inv, 12582912.0f);
+      q0 = low_clamp ? fmaxf(fminf(q0, 12582912.0f + 7.0f), 12582912.0f - 8.0f) : fminf(q0, 12582912.0f + 7.0f);
+      q1 = low_clamp ? fmaxf(fminf(q1, 12582912.0f + 7.0f), 12582912.0f - 8.0f) : fminf(q1, 12582912.0f + 7.0f);
+      // position j = h * 128 + 2p (even) and j + 1: lane h * 64 + p of the even / odd plane
+      even[h * (HD / 2) + p] = uint8_t(__float_as_uint(q0) << 4);
+      odd[h * (HD / 2) + p] = uint8_t(__float_as_uint(q1) << 4);
+    }
+  }
+  __syncthreads();
+  if (blockIdx.x == 0 && xq_out != nullptr) fused_export_codes(&xs[0][0][0], M, K, xq_out);
+  fused_products<CW>(&xs[0][0][0], sdx, red, w, group, groups, Wq, M, N, dw, Y, ldy);
 }
 
 }  // namespace
@@ -434,6 +476,33 @@ int smoothrot_linear_decode(const void* X_f16, int64_t M, int64_t K, int64_t ldx
     fused_plain_decode_kernel<1><<<grid, kFusedThreads, 0, st>>>(x, int(M), ldx, pre, clip_a, Wq, int(N), dw, y, ldy,
                                                                  Xq_out, dx_out);
   }
+  count_launch();
+  return launch_status();
+}
+
+int smoothrot_linear_decode_heads(const void* X_f16, int64_t M, int64_t n_heads, int64_t head_dim, int64_t ldx,
+                                  const float* pre, float clip_a, const uint8_t* Wq, const float* dw, int64_t N,
+                                  void* Y_f16, int64_t ldy, uint8_t* Xq_out, float* dx_out, void* stream) {
+  using namespace smoothrot;
+  using namespace smoothrot::gemm;
+  if (M < 0 || N < 0 || n_heads <= 0 || head_dim <= 0) return SMOOTHROT_INVALID_ARG;
+  if (!(clip_a > 0.0f) || clip_a > 1.0f) return SMOOTHROT_INVALID_ARG;
+  if (n_heads != 32 || head_dim != 128) return SMOOTHROT_UNSUPPORTED_K;
+  if (M > kFusedMaxTokens || N % 8 != 0 || N > 0x3fffffffLL) return SMOOTHROT_INVALID_ARG;
+  if (M == 0 || N == 0) return SMOOTHROT_OK;
+  const int64_t K = n_heads * head_dim;
+  if (X_f16 == nullptr || Wq == nullptr || dw == nullptr || Y_f16 == nullptr || ldx < K || ldy < N)
+    return SMOOTHROT_INVALID_ARG;
+  if (!aligned16(X_f16) || ldx % 8 != 0 || !aligned16(Wq) || (pre != nullptr && !aligned16(pre)))
+    return SMOOTHROT_BAD_ALIGNMENT;
+  const bool low = 7.0f / clip_a >= 8.49f;
+  const int64_t groups = (N + 15) / 16;
+  const int64_t slots = int64_t(device_sm_count()) * 2;
+  const int64_t per_cta = (groups + slots - 1) / slots;
+  const unsigned grid = unsigned((groups + per_cta - 1) / per_cta);
+  fused_heads_decode_kernel<<<grid, kFusedThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const __half*>(X_f16), int(M), ldx, pre, clip_a, low, Wq, int(N), dw, static_cast<__half*>(Y_f16), ldy,
+      Xq_out, dx_out);
   count_launch();
   return launch_status();
 }

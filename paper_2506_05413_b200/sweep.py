@@ -9,7 +9,7 @@ smoothrot_quant_act and smoothrot_linear, on seeded synthetic activations (rando
 weights, quantized once by smoothrot_fuse_weights), and prints time, TOP/s and GB/s; for the q/o
 shape also smoothrot_quant_act_heads (32 heads of 128), the transform the o-projection's input takes,
 and for K = 4096 smoothrot_linear_decode, which does both calls in one kernel (M <= 4 with the
-rotation: "fused"; M <= 8 without: "fusedP").
+rotation: "fused"; M <= 8 without: "fusedP"; M <= 4 with the head mixing, q/o shape: "fusedH").
 
 Timing: each call is recorded into a CUDA graph per buffer set and replayed back to back
 between two CUDA events; the buffer sets rotate so that their total size exceeds twice the
@@ -78,7 +78,7 @@ def run(reps: int = 30, shapes=None, tokens=None):
                 sr.linear(xq, dx, wq, dw, Y, ws)
                 sets.append((X, xq, dx, wq, dw, Y, ws))
             torch.cuda.synchronize()
-            gq, gl, gh, gf, gp, gfp = [], [], [], [], [], []
+            gq, gl, gh, gf, gp, gfp, gfh = [], [], [], [], [], [], []
             for X, xq, dx, wq, dw, Y, ws in sets:
                 sr.quant_act_plain(X, pre_x, case.clip_a, xq, dx)       # the quantizer without a rotation
                 g = torch.cuda.CUDAGraph()
@@ -91,6 +91,12 @@ def run(reps: int = 30, shapes=None, tokens=None):
                     with torch.cuda.graph(g):
                         sr.linear_decode(X, pre_x, case.clip_a, wq, dw, Y, rotation=False)
                     gfp.append(g)
+                if M <= 4 and name == "q_o":    # the o-projection's layer: head mixing + linear in one kernel
+                    sr.linear_decode_heads(X, HEADS, None, case.clip_a, wq, dw, Y)
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g):
+                        sr.linear_decode_heads(X, HEADS, None, case.clip_a, wq, dw, Y)
+                    gfh.append(g)
                 if M <= 4 and K == 4096:    # both calls of the layer in one kernel
                     sr.linear_decode(X, pre_x, case.clip_a, wq, dw, Y)
                     g = torch.cuda.CUDAGraph()
@@ -116,6 +122,7 @@ def run(reps: int = 30, shapes=None, tokens=None):
             tf = _time_graphs(torch, gf, reps) if gf else None
             tp = _time_graphs(torch, gp, reps)
             tfp = _time_graphs(torch, gfp, reps) if gfp else None
+            tfh = _time_graphs(torch, gfh, reps) if gfh else None
             tq = _time_graphs(torch, gq, reps)
             assert sr.device_status() == 0
             ops = 2.0 * M * N * K
@@ -133,6 +140,8 @@ def run(reps: int = 30, shapes=None, tokens=None):
                 rows[-1]["fused_layer_us"] = tf * 1e6
             if tfp is not None:
                 rows[-1]["fused_plain_layer_us"] = tfp * 1e6
+            if tfh is not None:
+                rows[-1]["fused_heads_layer_us"] = tfh * 1e6
             if th is not None:
                 rows[-1]["quant_act_heads_us"] = th * 1e6
                 rows[-1]["quant_act_heads_GBs"] = (2.5 * M * K + 4 * M) / th / 1e9
@@ -197,13 +206,14 @@ def main():
             print(json.dumps(r))
         return
     print(f"{'shape':8s} {'M':>5s} {'quant us':>9s} {'GB/s':>7s} {'plain us':>9s} {'GB/s':>7s} {'linear us':>10s} {'TOP/s':>8s} {'W GB/s':>8s}"
-          f" {'heads us':>9s} {'GB/s':>7s} {'fused us':>9s} {'fusedP us':>9s}")
+          f" {'heads us':>9s} {'GB/s':>7s} {'fused us':>9s} {'fusedP us':>9s} {'fusedH us':>9s}")
     for r in rows:
         heads = (f" {r['quant_act_heads_us']:9.1f} {r['quant_act_heads_GBs']:7.0f}"
                  if "quant_act_heads_us" in r else " " * 18)
         heads += f" {r['fused_layer_us']:9.1f}" if "fused_layer_us" in r else " " * 10
-        if "fused_plain_layer_us" in r:
-            heads += f" {r['fused_plain_layer_us']:9.1f}"
+        heads += f" {r['fused_plain_layer_us']:9.1f}" if "fused_plain_layer_us" in r else " " * 10
+        if "fused_heads_layer_us" in r:
+            heads += f" {r['fused_heads_layer_us']:9.1f}"
         print(f"{r['shape']:8s} {r['M']:5d} {r['quant_act_us']:9.1f} {r['quant_act_GBs']:7.0f} "
               f"{r['quant_act_plain_us']:9.1f} {r['quant_act_plain_GBs']:7.0f} "
               f"{r['linear_us']:10.1f} {r['linear_TOPS']:8.1f} {r['weight_stream_GBs']:8.0f}{heads}")

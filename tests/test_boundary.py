@@ -78,6 +78,11 @@ def test_host_side_rejections(lib):
     assert ld(dummy, 2, 4096, 4096, 1, None, 0.9, dummy, dummy, 12, dummy, 16, None, None, None) == -1    # N % 8
     assert ld(odd, 2, 4096, 4096, 0, None, 0.9, dummy, dummy, 16, dummy, 16, None, None, None) == -3
     assert ld(dummy, 0, 4096, 4096, 1, None, 0.9, dummy, dummy, 16, dummy, 16, None, None, None) == 0
+    ldh = lib.smoothrot_linear_decode_heads
+    assert ldh(dummy, 5, 32, 128, 4096, None, 0.9, dummy, dummy, 16, dummy, 16, None, None, None) == -1   # M > 4
+    assert ldh(dummy, 2, 16, 128, 2048, None, 0.9, dummy, dummy, 16, dummy, 16, None, None, None) == -2   # 32 x 128 only
+    assert ldh(dummy, 2, 32, 128, 4000, None, 0.9, dummy, dummy, 16, dummy, 16, None, None, None) == -1   # ldx < K
+    assert ldh(dummy, 0, 32, 128, 4096, None, 0.9, dummy, dummy, 16, dummy, 16, None, None, None) == 0
     lin = lib.smoothrot_linear
     assert lin(dummy, dummy, 4, dummy, dummy, 8, 100, dummy, 8, None, 0, None) == -2   # K % 128
     assert lin(dummy, dummy, 4, dummy, dummy, 12, 128, dummy, 16, None, 0, None) == -1  # N % 8

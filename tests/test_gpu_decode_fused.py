@@ -146,6 +146,41 @@ def test_fused_decode_without_rotation(gu, M, N, width, use_pre):
     assert np.array_equal(Y2.cpu().numpy(), Y)
 
 
+@pytest.mark.parametrize("M", [1, 2, 3, 4])
+@pytest.mark.parametrize("N", [4096, 1000, 14336])
+@pytest.mark.parametrize("use_pre", [False, True])
+def test_fused_decode_with_the_head_mixing_transform(gu, M, N, use_pre):
+    """smoothrot_linear_decode_heads: the tokens take smoothrot_quant_act_heads' path (32 heads of 128)."""
+    import torch
+    from paper_2506_05413_b200 import binding as sr
+    X = _acts(7 * M + N, M)
+    rng = np.random.default_rng(N + 1)
+    pre = (rng.uniform(0.05, 4.0, K) * (rng.integers(0, 2, K) * 2 - 1)).astype(np.float32) if use_pre else None
+    wq, dw = _weights(N + 2 * M, N)
+    pre_d = gu.dev(pre) if pre is not None else None
+    Y = torch.full((M, N), float("nan"), dtype=torch.float16, device=gu.DEV)
+    xq = torch.full((M, K // 2), 0x5A, dtype=torch.uint8, device=gu.DEV)
+    dx = torch.full((M,), float("nan"), dtype=torch.float32, device=gu.DEV)
+    sr.linear_decode_heads(gu.dev(X), 32, pre_d, 0.9, gu.dev(wq), gu.dev(dw), Y, xq, dx)
+    torch.cuda.synchronize()
+    Yh, xqh, dxh = Y.cpu().numpy(), xq.cpu().numpy(), dx.cpu().numpy()
+    q_ref, step_ref, _ = orc.quant_act_heads(X, pre, 32, 0.9)
+    assert np.abs(dxh / step_ref - 1).max() <= TOL_SCALE
+    frac, worst = gu.code_mismatch(xqh, q_ref)
+    assert worst <= 1 and frac <= max(TOL_CODES, 1.5 / xqh.size / 2)
+    assert np.isfinite(Yh.astype(np.float32)).all()
+    assert gu.rowwise_rel(Yh, orc.linear(xqh, dxh, wq, dw)) <= TOL_OUT
+    # the two-call path (same arithmetic, call by call) gives the same codes and outputs
+    q2 = torch.empty((M, K // 2), dtype=torch.uint8, device=gu.DEV)
+    s2 = torch.empty(M, dtype=torch.float32, device=gu.DEV)
+    Y2 = torch.empty((M, N), dtype=torch.float16, device=gu.DEV)
+    sr.quant_act_heads(gu.dev(X), 32, pre_d, 0.9, q2, s2)
+    sr.linear(q2, s2, gu.dev(wq), gu.dev(dw), Y2)
+    torch.cuda.synchronize()
+    assert np.array_equal(q2.cpu().numpy(), xqh) and np.array_equal(s2.cpu().numpy(), dxh)
+    assert np.array_equal(Y2.cpu().numpy(), Yh)
+
+
 def test_fused_decode_rejects_what_it_does_not_cover(gu):
     import torch
     from paper_2506_05413_b200 import binding as sr
