@@ -102,8 +102,8 @@ int smoothrot_fuse_weights(const void* W_f16, int64_t N, int64_t K, int64_t ldw,
 
 /*
  * Offline weight path with the clip-ratio search of the paper's weight quantizer (Experimental
- * settings, "Quantization": per-channel symmetric weights whose "clipping ratios [are] determined
- * through a linear search over the squared error").  As smoothrot_fuse_weights, but for every row
+ * settings, "Quantization": per-channel symmetric weights; each clip ratio is the candidate with the
+ * least squared quantization error, the candidates being tried one after another).  As smoothrot_fuse_weights, but for every row
  * the ratio is chosen from the grid
  *     ratio_i = fp32(1 - i * (1 - lowest_ratio) / (ratio_count - 1)),   i = 0 .. ratio_count - 1
  * (the paper gives no grid; 1.00 .. 0.50 in 51 steps is what the tests and the oracle use) as the
@@ -137,8 +137,8 @@ int smoothrot_quant_act(const void* X_f16, int64_t M, int64_t K, int64_t ldx,
 
 /*
  * Online activation quantizer of the layers that have no online Hadamard transform.  Methodology
- * section, last paragraph: online quantization is integrated into the forward pass for the
- * activations, while only two Hadamard transforms are (smoothrot_quant_act and
+ * section, last paragraph: every quantized layer quantizes its activations online, in the forward
+ * pass, while only two layers also rotate them there (smoothrot_quant_act and
  * smoothrot_quant_act_heads); every other quantized layer receives activations that are already
  * in the rotated basis.  For every token m:
  *     x^   = X[m][:] * pre                       (pre [K] fp32, or NULL for none)
@@ -150,9 +150,9 @@ int smoothrot_quant_act_plain(const void* X_f16, int64_t M, int64_t K, int64_t l
                               uint8_t* Xq_out, float* dx_out, void* stream);
 
 /*
- * Online activation path in front of the attention output projection.  Methodology section: "two
- * additional Hadamard transformations integrated into the forward pass, as described in [QuaRot]";
- * the paper spells out only the one before the down-projection (smoothrot_quant_act).  The other
+ * Online activation path in front of the attention output projection.  Methodology section: the
+ * forward pass contains two online Hadamard transforms, for which the paper defers to QuaRot; it
+ * spells out only the one before the down-projection (smoothrot_quant_act).  The other
  * one, as QuaRot describes it, mixes the heads of the attention output: a row of X is the
  * concatenation of n_heads head outputs of head_dim values, and
  *     x^[m][g * head_dim + e] = sum_h X[m][h * head_dim + e] * pre[h * head_dim + e] * H[h][g] / sqrt(n_heads)

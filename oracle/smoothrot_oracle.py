@@ -23,12 +23,12 @@ What follows the paper, by passage:
   quantization, group size 128 and clip ratio 0.95 (kv_quantize).
 * Fig. 2 (the feed-forward block): the down-projection input is the gated
   product sigma(gate) (.) up; quant_act_glu takes that edge in one step.
-* Section "Methodology", last paragraph: "online quantization operations are
-  integrated into the forward pass for [...] activations": the layers without
-  an online Hadamard transform quantize their input as it is (quant_act_plain).
-* Section "Methodology", "two additional Hadamard transformations integrated
-  into the forward pass, as described in [QuaRot]": the paper details the one
-  in front of the down-projection only.  The other sits in front of the
+* Section "Methodology", last paragraph: activations are quantized online, in
+  the forward pass, for every quantized layer; the layers without an online
+  Hadamard transform quantize their input as it is (quant_act_plain).
+* Section "Methodology": the forward pass contains two online Hadamard
+  transforms, for which the paper defers to QuaRot; it details the one in
+  front of the down-projection only.  The other sits in front of the
   attention output projection and, as QuaRot describes it, mixes the heads:
   (H_heads (x) I_head_dim) / sqrt(heads), the per-head factor
   (I (x) H_head_dim) being folded into the value projection offline
@@ -346,8 +346,8 @@ def fuse_weights(W: np.ndarray, pre_w, K: int, clip_w: float = 1.0):
 
 def clip_ratios(count: int = 51, lowest: float = 0.5) -> np.ndarray:
     """The grid of the weight clip search: `count` ratios from 1.0 down to `lowest`, equally
-    spaced, as float32.  The paper only says that the ratio is found by a linear search over the
-    squared error; the grid is this repository's reading."""
+    spaced, as float32.  The paper only says that each ratio is the one with the least squared
+    quantization error among candidates tried one after another; the grid is this repository's reading."""
     i = np.arange(count, dtype=np.float64)
     return (1.0 - i * (1.0 - lowest) / (count - 1)).astype(np.float32)
 
@@ -377,8 +377,8 @@ def clip_search_rows(v: np.ndarray, ratios: np.ndarray):
 
 def fuse_weights_search(W: np.ndarray, pre_w, K: int, ratios: np.ndarray):
     """Offline weight path with the clip-ratio search of the paper's weight quantizer
-    (Experimental settings, "Quantization": clipping ratios found by a linear search over the
-    squared error): rotate as in fuse_weights, then clip_search_rows per output channel.
+    (Experimental settings, "Quantization": the weight clip ratios are picked by least squared
+    error over a scan of candidates): rotate as in fuse_weights, then clip_search_rows per output channel.
     Returns (packed [N, K/2] u8, step [N] f32, best index [N], errors [N, len(ratios)], rotated f32)."""
     wr = rotate(W, pre_w, K).astype(np.float32)
     codes, step, best, errs = clip_search_rows(wr, ratios)

@@ -1,6 +1,6 @@
 // Weight quantization with the clip-ratio search of the paper's weight quantizer
-// (Experimental settings, "Quantization": per-channel symmetric 4-bit weights whose clipping
-// ratios are found by a linear search over the squared error).
+// (Experimental settings, "Quantization": per-channel symmetric 4-bit weights, each clip ratio
+// being the candidate with the least squared quantization error).
 //
 // Offline path, built for clarity rather than speed: the rows are rotated by the same kernels
 // as smoothrot_fuse_weights (through the fp32 export) into the caller's workspace, then one CTA

@@ -1,8 +1,8 @@
 // Head-mixing online transform of libsmoothrot:  v = (x * pre) (H_heads (x) I_head_dim) / sqrt(heads),
 // followed by the per-token symmetric 4-bit quantizer of the activation path.
 //
-// Methodology section: "two additional Hadamard transformations integrated into the forward pass, as
-// described in [QuaRot]".  The one in front of the down-projection is the full rotation of
+// Methodology section: the forward pass contains two online Hadamard transforms, for which the paper
+// defers to QuaRot.  The one in front of the down-projection is the full rotation of
 // rotate_quant.cu; this is the other one, in front of the attention output projection, where the
 // per-head factor of the rotation is folded into the value projection offline and only the mixing of
 // the heads is left for the forward pass.

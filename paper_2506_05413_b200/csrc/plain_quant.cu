@@ -1,8 +1,8 @@
 // Online activation quantizer without a rotation:  v = x * pre,  per-token symmetric INT4, packed.
 //
-// Methodology section, last paragraph: online quantization is part of the forward pass for the
-// activations of every quantized layer, while only two Hadamard transforms are (in front of the
-// down-projection and of the attention output projection).  The other layers see activations that
+// Methodology section, last paragraph: every quantized layer quantizes its activations online, in
+// the forward pass, while only two layers also rotate them there (the down-projection and the
+// attention output projection).  The other layers see activations that
 // are already in the rotated basis and only quantize them; this is that kernel.
 //
 // Pure streaming work, 2 bytes in and half a byte out per value: T threads share a row, a thread

@@ -1,5 +1,5 @@
 """Pins for the oracle's weight clip-ratio search (Experimental settings, "Quantization":
-a linear search over the squared error).  CPU only."""
+the ratio with the least squared quantization error among a scan of candidates).  CPU only."""
 import numpy as np
 
 from oracle import smoothrot_oracle as orc
