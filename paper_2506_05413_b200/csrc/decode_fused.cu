@@ -30,6 +30,29 @@ constexpr int kFusedChunksPerWarp = kFusedK / 128 / kFusedWarps;   // 64-byte ch
 
 __device__ __forceinline__ int padded(int j) { return j + (j >> 4); }
 
+// Thread-block cluster helpers: rank and size of the cluster, the address of one of this CTA's
+// shared-memory locations in another CTA of the cluster, the two halves of the cluster barrier.
+__device__ __forceinline__ uint32_t fused_cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t fused_cluster_size() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t fused_peer_address(const void* own, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;"
+               : "=r"(r) : "r"(uint32_t(__cvta_generic_to_shared(own))), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void fused_cluster_arrive() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void fused_cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+
 // Four butterfly stages between 16 values held by one thread.
 __device__ __forceinline__ void butterflies16(float (&v)[16]) {
 #pragma unroll
@@ -163,9 +186,13 @@ fused_decode_kernel(const __half* __restrict__ X, int M, int64_t ldx, const floa
 #pragma unroll
   for (int k = 0; k < 4; ++k)
     scale[k] = pre != nullptr ? __ldg(reinterpret_cast<const float4*>(pre + tid * 16) + k) : make_float4(1.f, 1.f, 1.f, 1.f);
+  // With several tokens the CTAs of a cluster divide them (token m is rotated by the CTA of rank
+  // m mod size) and fetch each other's codes through the cluster's shared-memory window afterwards.
+  const uint32_t crank = fused_cluster_rank(), csize = fused_cluster_size();
 #pragma unroll
   for (int m = 0; m < kFusedMaxTokens; ++m) {
     if (m >= M) break;
+    if (uint32_t(m) % csize != crank) continue;
     float v[16];
     {
       const uint4 a = raw_all[m][0], b = raw_all[m][1];
@@ -226,10 +253,35 @@ fused_decode_kernel(const __half* __restrict__ X, int M, int64_t ldx, const floa
     // the next token's first write to sred comes after two more barriers; buf is free since the barrier above
   }
   __syncthreads();
+  if (csize > 1) {
+    fused_cluster_arrive();               // this CTA's tokens are in its shared memory ...
+    fused_cluster_wait();                 // ... and so are everybody else's
+    for (int m = 0; m < M; ++m) {
+      const uint32_t owner = uint32_t(m) % csize;
+      if (owner == crank) continue;
+      const uint32_t src = fused_peer_address(&xs[m][0][0], owner);
+      uint4* dst = reinterpret_cast<uint4*>(&xs[m][0][0]);
+      for (int i = tid; i < 2 * (K / 8) / 4; i += kFusedThreads) {
+        uint4 val;
+        asm volatile("ld.shared::cluster.v4.b32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w) : "r"(src + uint32_t(i) * 16u) : "memory");
+        dst[i] = val;
+      }
+      if (tid == 0) {
+        float st;
+        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(st) : "r"(fused_peer_address(&sdx[m], owner)) : "memory");
+        sdx[m] = st;
+        if (blockIdx.x == 0 && dx_out != nullptr) dx_out[m] = st;
+      }
+    }
+    __syncthreads();
+    fused_cluster_arrive();               // done reading the others' shared memory (waited for before leaving)
+  }
   if (blockIdx.x == 0 && xq_out != nullptr) fused_export_codes(&xs[0][0][0], M, K, xq_out);
 
   // 3. the products, row group after row group
   fused_products<kFusedChunksPerWarp>(&xs[0][0][0], sdx, red, w, group, groups, Wq, M, N, dw, Y, ldy);
+  if (csize > 1) fused_cluster_wait();    // nobody leaves while its shared memory may still be read
 }
 
 // The same layer for inputs that need no online rotation (every quantized layer quantizes its input
@@ -464,8 +516,32 @@ int smoothrot_linear_decode(const void* X_f16, int64_t M, int64_t K, int64_t ldx
   __half* y = static_cast<__half*>(Y_f16);
   if (rotation) {
     const bool low = 7.0f / clip_a >= 8.49f;             // codes below -8 can only come up then
-    fused_decode_kernel<<<grid, kFusedThreads, 0, st>>>(x, int(M), ldx, pre, clip_a, low, Wq, int(N), dw, y, ldy,
-                                                        Xq_out, dx_out);
+    // several tokens: clusters of 2 or 4 CTAs share the rotations (the grid is rounded up to whole
+    // clusters; a CTA without row groups still rotates its tokens for the others)
+    const unsigned cs = M >= 3 ? 4u : (M == 2 ? 2u : 1u);
+    if (cs > 1) {
+      cudaLaunchConfig_t cfg{};
+      cfg.gridDim = dim3((grid + cs - 1) / cs * cs, 1, 1);
+      cfg.blockDim = dim3(kFusedThreads, 1, 1);
+      cfg.dynamicSmemBytes = 0;
+      cfg.stream = st;
+      cudaLaunchAttribute attr{};
+      attr.id = cudaLaunchAttributeClusterDimension;
+      attr.val.clusterDim.x = cs;
+      attr.val.clusterDim.y = 1;
+      attr.val.clusterDim.z = 1;
+      cfg.attrs = &attr;
+      cfg.numAttrs = 1;
+      const int m_int = int(M), n_int = int(N);
+      if (cudaLaunchKernelEx(&cfg, fused_decode_kernel, x, m_int, ldx, pre, clip_a, low, Wq, n_int, dw, y, ldy, Xq_out,
+                             dx_out) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return SMOOTHROT_CUDA_ERROR;
+      }
+    } else {
+      fused_decode_kernel<<<grid, kFusedThreads, 0, st>>>(x, int(M), ldx, pre, clip_a, low, Wq, int(N), dw, y, ldy,
+                                                          Xq_out, dx_out);
+    }
   } else if (K == 4096) {
     fused_plain_decode_kernel<4><<<grid, kFusedThreads, 0, st>>>(x, int(M), ldx, pre, clip_a, Wq, int(N), dw, y, ldy,
                                                                  Xq_out, dx_out);
