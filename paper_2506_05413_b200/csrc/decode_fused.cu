@@ -309,16 +309,17 @@ fused_plain_decode_kernel(const __half* __restrict__ X, int M, int64_t ldx, cons
   const int group = blockIdx.x;
   if (group < groups) fused_load_weights<CW>(w, Wq, N, group, warp, g, t);
 
-  // all tokens' values are requested at once: one trip to L2 instead of one per token
-  uint4 raw_all[kTokens][kPerThread];
-#pragma unroll
-  for (int m = 0; m < kTokens; ++m)
+  // a token's values are requested while the token before it is quantized (the loop over the tokens
+  // is kept rolled: unrolled, every token runs its own copy of the code and waits for it to be fetched)
+  auto fetch = [&](uint4 (&raw)[kPerThread], int m) {
 #pragma unroll
     for (int i = 0; i < kPerThread; ++i) {
       const int c = tid + i * kFusedThreads;
-      raw_all[m][i] = (m < M && c < kChunks) ? __ldg(reinterpret_cast<const uint4*>(X + int64_t(m) * ldx) + c)
-                                             : make_uint4(0u, 0u, 0u, 0u);
+      raw[i] = c < kChunks ? __ldg(reinterpret_cast<const uint4*>(X + int64_t(m) * ldx) + c) : make_uint4(0u, 0u, 0u, 0u);
     }
+  };
+  uint4 raw_next[kPerThread];
+  fetch(raw_next, 0);
   // the diagonal of this thread's chunks, once for all tokens
   f32x2 scale[kPerThread][4];
 #pragma unroll
@@ -334,14 +335,17 @@ fused_plain_decode_kernel(const __half* __restrict__ X, int M, int64_t ldx, cons
     scale[i][2] = pack2(b.x, b.y);
     scale[i][3] = pack2(b.z, b.w);
   }
+#pragma unroll 1
+  for (int m = 0; m < M; ++m) {
+    uint4 raw_cur[kPerThread];
 #pragma unroll
-  for (int m = 0; m < kTokens; ++m) {
-    if (m >= M) break;
+    for (int i = 0; i < kPerThread; ++i) raw_cur[i] = raw_next[i];
+    if (m + 1 < M) fetch(raw_next, m + 1);
     f32x2 v[kPerThread][4];
     float amax = 0.0f;
 #pragma unroll
     for (int i = 0; i < kPerThread; ++i) {
-      const uint4 raw = raw_all[m][i];
+      const uint4 raw = raw_cur[i];
       v[i][0] = half2_to_f32x2(raw.x);
       v[i][1] = half2_to_f32x2(raw.y);
       v[i][2] = half2_to_f32x2(raw.z);
