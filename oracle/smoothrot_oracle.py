@@ -23,6 +23,9 @@ What follows the paper, by passage:
   quantization, group size 128 and clip ratio 0.95 (kv_quantize).
 * Fig. 2 (the feed-forward block): the down-projection input is the gated
   product sigma(gate) (.) up; quant_act_glu takes that edge in one step.
+* Fig. 2 and section "Methodology": the whole feed-forward block, with
+  Lambda^-1 absorbed into the up-projection and Lambda into the
+  down-projection (absorb_into_up, ffn_block and their float64 companions).
 * Section "Methodology", last paragraph: activations are quantized online, in
   the forward pass, for every quantized layer; the layers without an online
   Hadamard transform quantize their input as it is (quant_act_plain).
@@ -470,6 +473,87 @@ def quant_act_glu(gate: np.ndarray, up: np.ndarray, pre_x, K: int, clip_a: float
     xr = rotate(glu_product(gate, up), pre_x, K).astype(np.float32)
     codes, step = quantize_rows(xr, clip_a)
     return pack_codes(codes), step, xr
+
+
+# ---------------------------------------------------------------------------
+# The feed-forward block of Fig. 2: up/gate projection -> sigma(gate) (.) up ->
+# hadamard -> quantize -> down projection, with Lambda^-1 in the up-projection
+# and Lambda in the down-projection (section "Methodology").
+# ---------------------------------------------------------------------------
+
+def absorb_into_up(W_up: np.ndarray, s: np.ndarray) -> np.ndarray:
+    """Lambda^-1 absorbed into the up-projection (section "Methodology": the smoothing diagonal
+    of the down-projection input goes into the up-projection, which is legal because the gated
+    product is taken channel by channel): output channel j of W_up ([I, K1], rows = the
+    down-projection's input channels) is divided by s_j.  float64, not rounded."""
+    return np.asarray(W_up, dtype=np.float64) / np.asarray(s, dtype=np.float64)[:, None]
+
+
+def ffn_plain_fp64(X, W_gate, W_up, W_down) -> np.ndarray:
+    """(SiLU(X W_gate^T) (.) X W_up^T) W_down^T: the block of Fig. 2 without any transformation
+    or quantization, float64."""
+    X = np.asarray(X, np.float64)
+    h = glu_product(X @ np.asarray(W_gate, np.float64).T, X @ np.asarray(W_up, np.float64).T)
+    return h @ np.asarray(W_down, np.float64).T
+
+
+def ffn_transformed_fp64(X, W_gate, W_up, W_down, s, d) -> np.ndarray:
+    """The same block after the method's transformation and before any quantization, float64:
+    the up-projection carries Lambda^-1 (absorb_into_up), the gated product is multiplied by the
+    sign diagonal d and rotated online by H / sqrt(I), and the down-projection's rows carry
+    Lambda, d and the same rotation (fuse_weights' map).  By Eq. 2, applied through the
+    channel-wise product, this equals ffn_plain_fp64 in exact arithmetic."""
+    X = np.asarray(X, np.float64)
+    I = np.asarray(W_down).shape[1]
+    d64 = np.ones(I) if d is None else np.asarray(d, np.float64)
+    h = glu_product(X @ np.asarray(W_gate, np.float64).T, X @ absorb_into_up(W_up, s).T)
+    hr = rotate(h, d64, I)
+    wr = rotate(np.asarray(W_down, np.float64), np.asarray(s, np.float64) * d64, I)
+    return hr @ wr.T
+
+
+def ffn_calibrate(X_calib, W_gate, W_up, W_down, alpha: float):
+    """Smoothing scales of the down-projection: the calibration set is sent through the
+    unquantized gate/up projections in float64, the gated products are rounded once to fp16 (the
+    dtype calibration inputs are handed over in) and enter `calibrate` with the original W_down.
+    Returns (h_calib fp16 [T, I], amax [I], s [I])."""
+    Xc = np.asarray(X_calib, np.float64)
+    h = glu_product(Xc @ np.asarray(W_gate, np.float64).T, Xc @ np.asarray(W_up, np.float64).T)
+    with np.errstate(over="ignore"):
+        h16 = np.clip(h, -65504.0, 65504.0).astype(np.float16)
+    amax, s = calibrate(h16, W_down, alpha)
+    return h16, amax, s
+
+
+def ffn_block(X, W_gate, W_up, W_down, s, d, clip_a: float = 0.9, clip_w: float = 1.0):
+    """The quantized feed-forward block of Fig. 2, every arrow one step of this file:
+
+        W_up'  = fp16(absorb_into_up(W_up, s))                 (weights are stored in fp16)
+        gate/up layer:  quant_act(X, None, K1) -> linear with fuse_weights([W_gate; W_up'], None, K1)
+                        -> G, U  fp16 [M, I]   (one fused layer of 2 I output channels)
+        x -> hadamard -> quantize:  quant_act_glu(G, U, d, I)  (Lambda^-1 already sits in W_up')
+        down layer:  linear with fuse_weights(W_down, s * d, I)
+
+    The block input is rotated online by the order-K1 Hadamard matrix and the gate/up weights
+    carry the same rotation, which stands in for the residual-stream rotation the paper folds
+    into the neighbouring layers offline.  Returns a dict of every intermediate."""
+    X = np.asarray(X)
+    K1 = X.shape[1]
+    I = np.asarray(W_down).shape[1]
+    with np.errstate(over="ignore"):
+        W_up_abs = absorb_into_up(W_up, s).astype(np.float16)
+    W_gu = np.concatenate([np.asarray(W_gate, np.float16), W_up_abs], axis=0)
+    wq_gu, dw_gu, _ = fuse_weights(W_gu, None, K1, clip_w)
+    xq, dx, _ = quant_act(X, None, K1, clip_a)
+    Y_gu = linear(xq, dx, wq_gu, dw_gu)
+    G, U = Y_gu[:, :I], Y_gu[:, I:]
+    d32 = None if d is None else np.asarray(d, np.float32)
+    hq, dh, hr = quant_act_glu(G, U, d32, I, clip_a)
+    pre_w = np.asarray(s, np.float64) * (1.0 if d is None else np.asarray(d, np.float64))
+    wq_d, dw_d, _ = fuse_weights(W_down, pre_w.astype(np.float32), I, clip_w)
+    Y = linear(hq, dh, wq_d, dw_d)
+    return dict(W_up_abs=W_up_abs, wq_gu=wq_gu, dw_gu=dw_gu, xq=xq, dx=dx, Y_gu=Y_gu,
+                hq=hq, dh=dh, hr=hr, pre_w=pre_w.astype(np.float32), wq_d=wq_d, dw_d=dw_d, Y=Y)
 
 
 def gemm_i32_numpy(xq: np.ndarray, wq: np.ndarray) -> np.ndarray:
