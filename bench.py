@@ -1,14 +1,15 @@
 #!/usr/bin/env python
 """Benchmark of the SmoothRot W4A4 linear layer on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg1|cfg2|cfg3]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3] [--per-config 0|1]
     python bench.py --impl reference ...        # the CPU oracle on the host cores
 
 One "step" is one pass of the whole path over one batch of seeded synthetic
 input: calibrate (per-channel absmax -> scales), fuse_weights (scale, rotate,
 quantize, pack W), quant_act (Hadamard + per-token INT4 quantize + pack X) and
 linear (INT4 x INT4 GEMM + dequant to fp16).  The headline value is the layer's
-2*M*N*K integer operations divided by the time of the whole step.
+2*M*N*K integer operations divided by the time of the whole step, on the
+largest single-GPU workload (the fused gate/up projection, 8192 x 28672 x 4096).
 
 The device-timed region keeps every input resident in HBM; between steps the
 loop rotates through several distinct buffer sets whose total size exceeds
@@ -16,9 +17,17 @@ twice the L2 capacity, so no step finds its inputs in L2.  A step is launched
 as two CUDA graphs recorded from the library calls, so that the Python cost of
 a launch (longer than some of the kernels) does not sit in the device timeline;
 a pair of events around the second graph times the GEMM kernel inside the
-timed region.  The end-to-end figure starts from pinned host buffers, makes the
-calls eagerly and ends with the output back on the host, with the copies
-inside the timed region.
+timed region.  After the K-step region the same region is repeated until half a
+second of device time has been timed ("sustained": mean and minimum per step).
+The end-to-end figure starts from pinned host buffers, makes the calls eagerly
+and ends with the output back on the host, with the copies inside the timed
+region.
+
+The same run also measures an INT8 yardstick on the same GPU (a library int8
+GEMM, 8192^3, burst and two seconds back to back) and, on one GPU, times every
+call of the other workloads (`per_config`: the fused QKV projection, the
+down-projection with the order-28 x Walsh-512 rotation, and a token-count sweep
+over the linear shapes of one decoder block), each with its own clock record.
 
 Prints exactly one JSON line on rank 0.
 """
@@ -27,6 +36,7 @@ from __future__ import annotations
 import argparse
 import json
 import os
+import re
 import subprocess
 import sys
 import threading
@@ -41,21 +51,20 @@ if ROOT not in sys.path:
 from paper_2506_05413_b200 import synth  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
-# DRAM bytes (read + write) of one launch of the GEMM kernel from an ncu capture, by (M, N, K);
-# absent (None in the output) for shapes that were not captured or after the kernel changed.
-LINEAR_TRAFFIC = {(2048, 6144, 4096): 16.85e6 + 0.04e6}   # operands from DRAM; Y (25.2 MB) still in L2 at kernel end
 NOMINAL_INT8_TOPS = 4500.0
 NOMINAL_BF16_TFLOPS = 2250.0
+NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 METRIC = "w4a4_smoothrot_linear_tops"
 UNIT = "TOPS"
+SWEEP_TOKENS = (1, 16, 128, 512, 2048)
 
 WORKLOADS = {
     "cfg0": (synth.config0, "configs[0]: tiny layer, X [64 x 128], W [256 x 128]"),
     "cfg1": (synth.config1, "configs[1]: LLaMA-3.1-8B-shaped fused QKV, X [2048 x 4096], W [6144 x 4096]"),
     "cfg2": (synth.config2, "configs[2]: down_proj with online Hadamard, X [2048 x 14336], W [4096 x 14336]"),
-    "cfg3": (synth.config3, "configs[3]: fused gate/up, X [8192 x 4096], W [28672 x 4096]"),
+    "cfg3": (synth.config3, "configs[3]: fused gate/up projection (compute-bound GEMM), X [8192 x 4096], W [28672 x 4096]"),
 }
 
 
@@ -67,6 +76,24 @@ def measured_peaks():
         return dict(hbm_gbs=float(p["hbm_gbs"]), bf16=float(p["bf16_tflops"]),
                     bf16_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
     return dict(hbm_gbs=FALLBACK_HBM_GBS, bf16=FALLBACK_BF16_TFLOPS, bf16_sustained=1400.0, source="fallback")
+
+
+def profiled_traffic(M, N, K):
+    """DRAM bytes (read + write) per launch of the GEMM kernel for this shape, from the tracked ncu
+    summaries: a line `dram_bytes_per_launch M=.. N=.. K=..: <bytes>` in a file under profiles/.
+    None when no summary covers the shape."""
+    pat = re.compile(r"dram_bytes_per_launch\s+M=(\d+)\s+N=(\d+)\s+K=(\d+):\s*([0-9.eE+]+)")
+    folder = os.path.join(ROOT, "profiles")
+    if not os.path.isdir(folder):
+        return None
+    for name in sorted(os.listdir(folder)):
+        if not name.endswith((".md", ".txt")):
+            continue
+        with open(os.path.join(folder, name)) as f:
+            for m in pat.finditer(f.read()):
+                if (int(m.group(1)), int(m.group(2)), int(m.group(3))) == (M, N, K):
+                    return float(m.group(4))
+    return None
 
 
 def layer_ops(M, N, K):
@@ -84,19 +111,22 @@ def algorithmic_bytes(M, N, K, T):
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    """Samples nvidia-smi clocks and throttle reasons while a timed region runs."""
 
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index: int):
+    def __init__(self, index: int, enabled: bool = True):
         self.index = index
+        self.enabled = enabled
         self.lines = []
         self.proc = None
         self.thread = None
 
     def start(self):
+        if not self.enabled:
+            return self
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.QUERY}",
@@ -104,26 +134,40 @@ class ClockSampler:
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
-            return
+            return self
         self.thread = threading.Thread(target=self._pump, daemon=True)
         self.thread.start()
+        return self
 
     def _pump(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.perf_counter(), line.strip()))
 
-    def stop(self):
+    def mark(self):
+        return time.perf_counter()
+
+    def stop(self, since=None, until=None):
+        """Summary of the samples taken between the two marks (all samples if none given)."""
+        if not self.enabled:
+            return None
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
+        time.sleep(0.12)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
+        return self.summary(since, until)
+
+    def summary(self, since=None, until=None):
         sm, smax, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in self.lines:
+        for stamp, line in list(self.lines):
+            if since is not None and stamp < since:
+                continue
+            if until is not None and stamp > until + 0.06:
+                continue
             parts = [x.strip() for x in line.split(",")]
             if len(parts) < 8:
                 continue
@@ -135,8 +179,8 @@ class ClockSampler:
                 if flag.lower().startswith("active"):
                     reasons.add(name)
         if not sm:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
-        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(smax)),
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_min_mhz": float(min(sm)), "sm_max_mhz": float(max(smax)),
                 "power_w_max": float(max(power)), "samples": len(sm), "reasons": sorted(reasons)}
 
 
@@ -197,10 +241,12 @@ def run_reference(args, case, desc):
 class DeviceSet:
     """One resident copy of a layer's inputs and outputs."""
 
-    def __init__(self, torch, sr, case, dev):
+    def __init__(self, torch, sr, case, dev, M=None):
         t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
-        M, N, K = case.M, case.N, case.K
-        self.X, self.Xc, self.W, self.d = t(case.X), t(case.X_calib), t(case.W), t(case.d)
+        M = case.M if M is None else M
+        N, K = case.N, case.K
+        self.M = M
+        self.X, self.Xc, self.W, self.d = t(case.X[:M]), t(case.X_calib), t(case.W), t(case.d)
         f32 = lambda n: torch.empty(n, dtype=torch.float32, device=dev)
         self.amax, self.s, self.pre_w, self.pre_x = f32(K), f32(K), f32(K), f32(K)
         self.wq = torch.empty((N, K // 2), dtype=torch.uint8, device=dev)
@@ -212,6 +258,10 @@ class DeviceSet:
 
     def nbytes(self):
         tensors = (self.X, self.Xc, self.W, self.wq, self.xq, self.Y)
+        return sum(x.numel() * x.element_size() for x in tensors)
+
+    def online_nbytes(self):
+        tensors = (self.X, self.wq, self.xq, self.Y)
         return sum(x.numel() * x.element_size() for x in tensors)
 
 
@@ -255,6 +305,179 @@ def capture(torch, fns):
         for fn in fns:
             fn()
     return g
+
+
+def time_replays(torch, graphs, min_seconds=0.2, reps=20, max_regions=4000):
+    """Replays the graphs round robin, `reps` replays per event-bracketed region, region after
+    region until `min_seconds` of device time have been timed.  Returns (mean, minimum) seconds
+    per replay over the regions and the number of regions."""
+    n = len(graphs)
+    for i in range(max(3, n)):
+        graphs[i % n].replay()
+    torch.cuda.synchronize()
+    per, total, k = [], 0.0, 0
+    while total < min_seconds and len(per) < max_regions:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            graphs[k % n].replay()
+            k += 1
+        e1.record()
+        torch.cuda.synchronize()
+        sec = e0.elapsed_time(e1) * 1e-3
+        per.append(sec / reps)
+        total += sec
+    return float(np.mean(per)), float(np.min(per)), len(per)
+
+
+def int8_yardstick(torch, dev, seconds=2.0):
+    """An int8 tensor-core GEMM from the vendor library on this GPU's own memory (8192^3, int32
+    accumulation): best of ten single calls ("burst") and the mean rate of calls back to back for
+    `seconds` ("sustained").  A yardstick for the roofline's denominator only; no part of the path."""
+    n = 8192
+    try:
+        a = torch.randint(-8, 8, (n, n), dtype=torch.int8, device=dev)
+        b = torch.randint(-8, 8, (n, n), dtype=torch.int8, device=dev)
+        for _ in range(3):
+            torch._int_mm(a, b)
+        torch.cuda.synchronize()
+        best = float("inf")
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); torch._int_mm(a, b); e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1) * 1e-3)
+        ops = 2.0 * n ** 3
+        calls, total = 0, 0.0
+        while total < seconds:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(20):
+                torch._int_mm(a, b)
+            e1.record()
+            torch.cuda.synchronize()
+            total += e0.elapsed_time(e1) * 1e-3
+            calls += 20
+        del a, b
+        return {"burst_tops": ops / best / 1e12, "sustained_tops": ops * calls / total / 1e12,
+                "how": f"library int8 GEMM {n}^3, best of 10 / {calls} calls back to back ({total:.1f} s)"}
+    except Exception as exc:   # the yardstick is optional: report why it is missing
+        return {"burst_tops": None, "sustained_tops": None, "how": f"unavailable: {type(exc).__name__}: {exc}"}
+
+
+def peaks_record(peaks, yard):
+    rec = {
+        "hbm_gbs": peaks["hbm_gbs"], "hbm_source": f"{peaks['source']} copy bandwidth", "hbm_nominal_gbs": NOMINAL_HBM_GBS,
+        "int8_from_bf16_burst": peaks["bf16"] * 2.0, "int8_from_bf16_sustained": peaks["bf16_sustained"] * 2.0,
+        "int8_nominal": NOMINAL_INT8_TOPS,
+        "int8_measured_in_run_burst": yard["burst_tops"], "int8_measured_in_run_sustained": yard["sustained_tops"],
+        "int8_measured_how": yard["how"],
+    }
+    return rec
+
+
+def linear_fracs(tops, rec):
+    out = {"of_bf16_burst_x2": tops / rec["int8_from_bf16_burst"],
+           "of_bf16_sustained_x2": tops / rec["int8_from_bf16_sustained"],
+           "of_nominal_4500": tops / rec["int8_nominal"]}
+    if rec["int8_measured_in_run_burst"]:
+        out["of_int8_measured_burst"] = tops / rec["int8_measured_in_run_burst"]
+        out["of_int8_measured_sustained"] = tops / rec["int8_measured_in_run_sustained"]
+    return out
+
+
+def measure_layer(torch, sr, case, dev, rec, local, min_seconds, sampler_on=True):
+    """Every call of the path on one workload, each alone (graph replays, buffer sets rotated out
+    of L2), plus the whole step; with a clock record of its own."""
+    M, N, K, T = case.M, case.N, case.K, case.X_calib.shape[0]
+    first = DeviceSet(torch, sr, case, dev)
+    n_sets = max(2, int(np.ceil(2.2 * L2_BYTES / first.nbytes())))
+    sets = [first] + [DeviceSet(torch, sr, case, dev) for _ in range(1, n_sets)]
+    for ds in sets:
+        gpu_step(sr, case, ds)
+    torch.cuda.synchronize()
+    graphs = {name: [] for name in CALLS}
+    whole = []
+    for ds in sets:
+        calls = step_calls(sr, case, ds)
+        for name in CALLS:
+            graphs[name].append(capture(torch, [calls[name]]))
+        whole.append(capture(torch, [calls[name] for name in CALLS]))
+    sampler = ClockSampler(local, sampler_on).start()
+    abytes = algorithmic_bytes(M, N, K, T)
+    out = {"M": M, "N": N, "K": K, "buffer_sets": n_sets, "linear_kernel": sr.linear_plan_name(M, N, K)}
+    for name in CALLS:
+        mean, best, regions = time_replays(torch, graphs[name], min_seconds)
+        entry = {"us": mean * 1e6, "us_min": best * 1e6, "regions": regions,
+                 "GB/s": abytes[name] / mean / 1e9, "frac_hbm": abytes[name] / mean / 1e9 / rec["hbm_gbs"]}
+        if name == "linear":
+            tops = layer_ops(M, N, K) / mean / 1e12
+            entry["TOPS"] = tops
+            entry["frac"] = linear_fracs(tops, rec)
+        out[name] = entry
+    mean, best, regions = time_replays(torch, whole, min_seconds)
+    out["step"] = {"us": mean * 1e6, "us_min": best * 1e6, "TOPS": layer_ops(M, N, K) / mean / 1e12}
+    out["clocks"] = sampler.stop()
+    assert sr.device_status() == 0, "a device-side wait timed out"
+    del graphs, whole, sets, first
+    torch.cuda.empty_cache()
+    return out
+
+
+def measure_sweep(torch, sr, dev, rec, local, min_seconds, sampler_on=True):
+    """The online calls (quant_act, linear) of every linear shape of one decoder block at several
+    token counts, from decode to prefill; weights quantized once per shape; inputs, codes, weights
+    and outputs rotated out of L2."""
+    rows = []
+    for name, N, K in synth.BLOCK_SHAPES:
+        case = synth.config4(name, max(SWEEP_TOKENS))     # rows 0..M-1 of one draw serve every M
+        full = DeviceSet(torch, sr, case, dev)
+        gpu_step(sr, case, full)
+        torch.cuda.synchronize()
+        sampler = ClockSampler(local, sampler_on).start()
+        shape_rows = []
+        for M in SWEEP_TOKENS:
+            per_set = N * K // 2 + M * K * 2 + M * K // 2 + M * N * 2
+            n_sets = int(min(24, max(2, np.ceil(2.2 * L2_BYTES / per_set))))
+            sets = []
+            for _ in range(n_sets):
+                X = full.X[:M].clone()
+                wq, dw = full.wq.clone(), full.dw.clone()
+                xq = torch.empty((M, K // 2), dtype=torch.uint8, device=dev)
+                dx = torch.empty(M, dtype=torch.float32, device=dev)
+                Y = torch.empty((M, N), dtype=torch.float16, device=dev)
+                need = sr.workspace_bytes(M, N, K)
+                ws = torch.empty(need, dtype=torch.uint8, device=dev) if need else None
+                sr.quant_act(X, full.pre_x, case.clip_a, xq, dx)
+                sr.linear(xq, dx, wq, dw, Y, ws)
+                sets.append((X, xq, dx, wq, dw, Y, ws))
+            torch.cuda.synchronize()
+            gq = [capture(torch, [lambda s=s: sr.quant_act(s[0], full.pre_x, case.clip_a, s[1], s[2])]) for s in sets]
+            gl = [capture(torch, [lambda s=s: sr.linear(s[1], s[2], s[3], s[4], s[5], s[6])]) for s in sets]
+            tq, tq_min, _ = time_replays(torch, gq, min_seconds)
+            tl, tl_min, _ = time_replays(torch, gl, min_seconds)
+            ops = layer_ops(M, N, K)
+            row = {"shape": name, "N": N, "K": K, "M": M, "buffer_sets": n_sets,
+                   "linear_kernel": sr.linear_plan_name(M, N, K),
+                   "quant_act_us": tq * 1e6, "quant_act_us_min": tq_min * 1e6,
+                   "quant_act_GBs": (2.5 * M * K + 4 * M + 4 * K) / tq / 1e9,
+                   "linear_us": tl * 1e6, "linear_us_min": tl_min * 1e6, "linear_TOPS": ops / tl / 1e12,
+                   "linear_frac_bf16_burst_x2": ops / tl / 1e12 / rec["int8_from_bf16_burst"],
+                   "weight_stream_GBs": 0.5 * N * K / tl / 1e9,
+                   "weight_stream_frac_hbm": 0.5 * N * K / tl / 1e9 / rec["hbm_gbs"],
+                   "algorithmic": {"ops": ops, "linear_bytes": 0.5 * M * K + 0.5 * N * K + 2.0 * M * N + 4.0 * (M + N),
+                                   "quant_act_bytes": 2.5 * M * K + 4 * M + 4 * K}}
+            shape_rows.append(row)
+            del sets, gq, gl
+            torch.cuda.empty_cache()
+        clocks = sampler.stop()
+        for row in shape_rows:
+            row["clocks"] = clocks
+        rows.extend(shape_rows)
+        assert sr.device_status() == 0, "a device-side wait timed out"
+        del full
+        torch.cuda.empty_cache()
+    return rows
 
 
 def run_gpu(args, case, desc):
@@ -313,43 +536,54 @@ def run_gpu(args, case, desc):
         back[i % n_sets].replay()
     torch.cuda.synchronize()
 
-    # ---- device-timed region: K steps ------------------------------------------------
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-    barrier()
-    start.record()
-    for i in range(args.steps):
-        front[i % n_sets].replay()
-        ev[i][0].record()
-        back[i % n_sets].replay()
-        ev[i][1].record()
-    stop.record()
-    barrier()
+    def timed_region(steps, with_events):
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)] if with_events else None
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        start.record()
+        for i in range(steps):
+            front[i % n_sets].replay()
+            if with_events:
+                ev[i][0].record()
+            back[i % n_sets].replay()
+            if with_events:
+                ev[i][1].record()
+        stop.record()
+        barrier()
+        total_ms = max_over_ranks(torch, dist, start.elapsed_time(stop), dev)
+        lin = float(np.mean([a.elapsed_time(b) for a, b in ev])) if with_events else None
+        return total_ms, lin
+
+    # ---- device-timed region: exactly K steps ---------------------------------------
+    sampler = ClockSampler(local, rank == 0).start()
+    t_a = sampler.mark()
+    total_ms, linear_live_ms = timed_region(args.steps, True)
+    t_b = sampler.mark()
     launches = launches_per_step * args.steps
-    clocks = sampler.stop() if rank == 0 else None
-    total_ms = max_over_ranks(torch, dist, start.elapsed_time(stop), dev)
     ms_per_step = total_ms / args.steps
-    linear_live_ms = float(np.mean([ev[i][0].elapsed_time(ev[i][1]) for i in range(args.steps)]))
     assert sr.device_status() == 0, "a device-side wait timed out"
 
+    # ---- the same region again and again until half a second of device time is covered ----
+    regions, covered = [ms_per_step], total_ms
+    while covered < args.min_region_s * 1e3 and len(regions) < 2000:
+        t_ms, _ = timed_region(args.steps, False)
+        regions.append(t_ms / args.steps)
+        covered += t_ms
+    t_c = sampler.mark()
+    # one record over the K-step region and its repeats (the same work; the first region alone can
+    # be shorter than the sampling interval), with the number of samples that fell into the first
+    clocks = sampler.stop(t_a, t_c) if rank == 0 else None
+    if clocks is not None:
+        clocks["samples_in_first_region"] = (sampler.summary(t_a, t_b) or {}).get("samples", 0)
+        clocks["covers"] = "the K-step region and its repeats (sustained)"
+
     # ---- each call alone (outside the timed region): one graph per call and buffer set ----
-    call_ms = {}
-    reps = max(10, min(args.steps, 100))
+    call_ms, call_ms_min = {}, {}
+    sampler2 = ClockSampler(local, rank == 0).start()
     for name in CALLS:
-        gs = single[name]
-        for i in range(3):
-            gs[i % n_sets].replay()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        e0.record()
-        for i in range(reps):
-            gs[i % n_sets].replay()
-        e1.record()
-        torch.cuda.synchronize()
-        call_ms[name] = e0.elapsed_time(e1) / reps
+        mean, best, _ = time_replays(torch, single[name], 0.25 if name == "linear" else 0.1)
+        call_ms[name], call_ms_min[name] = mean * 1e3, best * 1e3
+    clocks_calls = sampler2.stop() if rank == 0 else None
     call_ms_alone_linear = call_ms["linear"]
     call_ms["linear"] = linear_live_ms
 
@@ -395,24 +629,35 @@ def run_gpu(args, case, desc):
     e2e_steps_run(e2e_steps)
     barrier()
     e2e_sec = max_over_ranks(torch, dist, (time.perf_counter() - t0) / e2e_steps, dev)
+    del host_in, host_Y
 
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
 
-    ops = layer_ops(M, N, K)
+    # ---- the denominators: measured copy bandwidth, bf16-derived and in-run int8 rates ----
     peaks = measured_peaks()
-    int8_peak = peaks["bf16"] * (NOMINAL_INT8_TOPS / NOMINAL_BF16_TFLOPS)
+    yard = int8_yardstick(torch, dev)
+    rec = peaks_record(peaks, yard)
+
+    ops = layer_ops(M, N, K)
+    int8_peak = rec["int8_from_bf16_burst"]
     abytes = algorithmic_bytes(M, N, K, T)
     dominant = max(call_ms, key=call_ms.get)
     if dominant == "linear":
         achieved = ops / (call_ms["linear"] * 1e-3) / 1e12
-        roofline = {"kernel": "w4a4_gemm_pair_tmem_kernel (smoothrot_linear)", "bound": "tensor", "achieved": achieved,
-                    "peak": int8_peak, "unit": "TOP/s", "frac": achieved / int8_peak, "traffic": LINEAR_TRAFFIC.get((M, N, K)),
+        traffic = profiled_traffic(M, N, K)
+        roofline = {"kernel": f"{sr.linear_plan_name(M, N, K)} (smoothrot_linear)", "bound": "tensor",
+                    "achieved": achieved, "peak": int8_peak, "unit": "TOP/s", "frac": achieved / int8_peak,
+                    "traffic": traffic,
+                    "traffic_note": ("dram read + write bytes of one launch from the ncu summary under profiles/; "
+                                     "part of Y may still sit in L2 when the kernel ends") if traffic else
+                                    "no ncu summary under profiles/ covers this shape",
+                    "algorithmic_ops": ops, "algorithmic_bytes": abytes["linear"],
                     "timed": "CUDA events around the kernel's launch inside the timed region, mean over the steps",
                     "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16']} TFLOP/s x 2 (nominal int8:bf16 ratio)",
-                    "frac_of_nominal_4500": achieved / NOMINAL_INT8_TOPS}
+                    "fracs": linear_fracs(achieved, rec)}
     else:
         achieved = abytes[dominant] / (call_ms[dominant] * 1e-3) / 1e9
         roofline = {"kernel": dominant, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
@@ -422,11 +667,28 @@ def run_gpu(args, case, desc):
     per_call = {}
     for name in CALLS:
         sec = call_ms[name] * 1e-3
-        per_call[name] = {"ms": call_ms[name], "GB/s": abytes[name] / sec / 1e9,
-                          "frac_hbm": abytes[name] / sec / 1e9 / peaks["hbm_gbs"]}
+        per_call[name] = {"ms": call_ms[name], "ms_min_alone": call_ms_min[name], "GB/s": abytes[name] / sec / 1e9,
+                          "frac_hbm": abytes[name] / sec / 1e9 / peaks["hbm_gbs"],
+                          "frac_hbm_nominal_8000": abytes[name] / sec / 1e9 / NOMINAL_HBM_GBS,
+                          "algorithmic_bytes": abytes[name]}
     per_call["linear"]["TOPS"] = ops / (call_ms["linear"] * 1e-3) / 1e12
     per_call["linear"]["frac_int8_peak"] = per_call["linear"]["TOPS"] / int8_peak
     per_call["linear"]["ms_alone"] = call_ms_alone_linear
+    per_call["clocks"] = clocks_calls
+
+    # ---- the other workloads, one GPU only (each with its own clock record) ----
+    per_config = None
+    if args.per_config and world == 1:
+        del front, back, single, sets, first
+        torch.cuda.empty_cache()
+        per_config = {}
+        for key in ("cfg1", "cfg2"):
+            if key == args.workload:
+                continue
+            maker, d2 = WORKLOADS[key]
+            per_config[key] = measure_layer(torch, sr, maker(), dev, rec, local, args.min_config_s)
+            per_config[key]["workload"] = d2
+        per_config["cfg4_sweep"] = measure_sweep(torch, sr, dev, rec, local, args.min_config_s)
 
     # ---- the oracle on this machine's host cores, bounded sample ----------------------
     Ms, Ns = oracle_sample_shape(case)
@@ -442,31 +704,47 @@ def run_gpu(args, case, desc):
                    "step": "calibrate + fuse_weights + quant_act + linear",
                    "launch": "each step replays two CUDA graphs recorded from the C-ABI calls "
                              "([calibrate, fuse_weights, quant_act], [linear])",
-                   "l2": f"inputs rotate through {n_sets} buffer sets ({n_sets * first.nbytes() / 2**20:.0f} MiB > 2 x L2)",
+                   "l2": f"inputs rotate through {n_sets} buffer sets ({n_sets * first_bytes(M, N, K, T) / 2**20:.0f} MiB > 2 x L2)",
                    "parallelism": "replicas only" if world > 1 else "1 GPU"},
         "clocks": clocks,
+        "sustained": {"ms_per_step_mean": float(np.mean(regions)), "ms_per_step_min": float(np.min(regions)),
+                      "regions": len(regions), "device_seconds": covered * 1e-3,
+                      "TOPS_mean": world * ops / (float(np.mean(regions)) * 1e-3) / 1e12},
         "e2e": {"value": world * ops / e2e_sec / 1e12, "unit": UNIT, "ms_per_step": e2e_sec * 1e3,
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
         "gpu_launches": int(launches),
         "roofline": roofline,
+        "peaks": rec,
         "cpu_baseline": {"value": cpu_value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
                          "sample": sample},
         "per_call": per_call,
         "online_only": {"ms": call_ms["quant_act"] + call_ms["linear"],
                         "TOPS": ops / ((call_ms["quant_act"] + call_ms["linear"]) * 1e-3) / 1e12},
     }
+    if per_config is not None:
+        line["per_config"] = per_config
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
 
 
+def first_bytes(M, N, K, T):
+    """Bytes of one buffer set (inputs, codes, output)."""
+    return 2 * M * K + 2 * T * K + 2 * N * K + N * K // 2 + M * K // 2 + 2 * M * N
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
-    ap.add_argument("--workload", choices=sorted(WORKLOADS), default="cfg1")
+    ap.add_argument("--workload", choices=sorted(WORKLOADS), default="cfg3")
+    ap.add_argument("--per-config", type=int, default=1, help="0: skip the records of the other workloads")
+    ap.add_argument("--min-region-s", type=float, default=0.5,
+                    help="device seconds the repeated K-step regions must cover")
+    ap.add_argument("--min-config-s", type=float, default=0.06,
+                    help="device seconds per timed call in the per-config records")
     args = ap.parse_args()
     maker, desc = WORKLOADS[args.workload]
     rank = int(os.environ.get("RANK", "0"))

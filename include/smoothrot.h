@@ -288,6 +288,11 @@ int smoothrot_linear_decode_heads(const void* X_f16, int64_t M, int64_t n_heads,
  * the same result. */
 size_t smoothrot_workspace_bytes(int64_t M, int64_t N, int64_t K);
 
+/* Host. Name of the kernel (or kernel pair) smoothrot_linear launches for this shape when it is
+ * given the workspace smoothrot_workspace_bytes reports: a static string, "none" for shapes the
+ * call rejects.  For reports and benchmarks; nothing is launched. */
+const char* smoothrot_linear_plan_name(int64_t M, int64_t N, int64_t K);
+
 /*
  * Test exports: values the fused kernels never write to memory.
  *   smoothrot_debug_hadamard: Y[m][:] = (X[m][:] * pre) H / sqrt(K) as fp32

@@ -36,6 +36,7 @@ SIGNATURES = {
     "smoothrot_linear_decode_heads": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _f32, _vp, _vp, _i64, _vp, _i64, _vp, _vp, _vp]),
     "smoothrot_linear_decode": (_int, [_vp, _i64, _i64, _i64, _int, _vp, _f32, _vp, _vp, _i64, _vp, _i64, _vp, _vp, _vp]),
     "smoothrot_workspace_bytes": (_sz, [_i64, _i64, _i64]),
+    "smoothrot_linear_plan_name": (ctypes.c_char_p, [_i64, _i64, _i64]),
     "smoothrot_debug_hadamard": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp]),
     "smoothrot_debug_hadamard_heads": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _vp, _vp]),
     "smoothrot_debug_gemm_i32": (_int, [_vp, _i64, _vp, _i64, _i64, _vp, _vp, _sz, _vp]),
@@ -228,6 +229,11 @@ def kv_dequant(q, step, zero, Y):
 
 def workspace_bytes(M, N, K) -> int:
     return int(load().smoothrot_workspace_bytes(int(M), int(N), int(K)))
+
+
+def linear_plan_name(M, N, K) -> str:
+    """Name of the kernel smoothrot_linear launches for this shape (host call, nothing runs)."""
+    return load().smoothrot_linear_plan_name(int(M), int(N), int(K)).decode()
 
 
 def _packed(t, name):

@@ -89,11 +89,10 @@ __device__ __forceinline__ void unpack8_f16(const uint4& raw, float* f) {
   }
 }
 
-// SiLU(g) * u, the gated product of Fig. 2, in fp32 (fast exponential and division: relative
-// error below 1e-6, far inside the rotation tolerance).  Large |g| is safe: exp(-g) = inf gives
-// g / inf = -0, exp(-g) = 0 gives g.
+// SiLU(g) * u, the gated product of Fig. 2, in fp32 with the library exponential and an IEEE
+// division (a few ulp).  Large |g| is safe: exp(-g) = inf gives g / inf = -0, exp(-g) = 0 gives g.
 __device__ __forceinline__ float glu_product(float g, float u) {
-  return __fdividef(g, 1.0f + __expf(-g)) * u;
+  return __fdiv_rn(g, 1.0f + expf(-g)) * u;
 }
 
 // ---------------------------------------------------------------------------

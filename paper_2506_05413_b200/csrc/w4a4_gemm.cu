@@ -1781,6 +1781,17 @@ int smoothrot_linear_static_scratch(const uint8_t* Xq, const float* dx, int64_t 
              need > 0 ? kStaticScratchBytes : 0, static_cast<cudaStream_t>(stream));
 }
 
+const char* smoothrot_linear_plan_name(int64_t M, int64_t N, int64_t K) {
+  if (M <= 0 || N <= 0 || K <= 0 || K % smoothrot::gemm::kWideRow != 0) return "none";
+  const smoothrot::gemm::Plan pl = smoothrot::gemm::make_plan(M, N, K);
+  if (pl.gemv) return "w4a4_decode_kernel";
+  if (pl.swapped) return pl.cluster ? "w4a4_gemm_stream_kernel (k-splits in a cluster)"
+                                    : (pl.splits > 1 ? "w4a4_gemm_stream_kernel + splitk_reduce_kernel"
+                                                     : "w4a4_gemm_stream_kernel");
+  if (pl.pair) return pl.splits > 1 ? "w4a4_gemm_pair_tmem_kernel + splitk_reduce_kernel" : "w4a4_gemm_pair_tmem_kernel";
+  return "w4a4_gemm_kernel";
+}
+
 size_t smoothrot_workspace_bytes(int64_t M, int64_t N, int64_t K) {
   if (M <= 0 || N <= 0 || K <= 0 || K % smoothrot::gemm::kWideRow != 0) return 0;
   const smoothrot::gemm::Plan pl = smoothrot::gemm::make_plan(M, N, K);

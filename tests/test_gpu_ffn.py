@@ -1,0 +1,170 @@
+"""The feed-forward block of Fig. 2 through the C-ABI, stage by stage against the oracle:
+
+    gate/up layer (one fused smoothrot_linear of 2 I output channels, Lambda^-1 absorbed into the
+    up half) -> smoothrot_quant_act_glu on the two fp16 halves (strided views of one output, the
+    sign diagonal only) -> down layer (smoothrot_linear on weights that carry Lambda, the signs
+    and the rotation).
+
+Staged parity: every oracle stage is fed the GPU's upstream outputs, at the tolerances stated for
+the single layer (steps 1e-6, codes 1e-4 off by one, accumulators exact, outputs 2e-3 of the row
+maximum).  Reduced sizes are compared in full; at the model's widths (4096 -> 2 x 14336 -> 4096)
+the oracle takes sampled whole rows."""
+import numpy as np
+import pytest
+
+from oracle import smoothrot_oracle as orc
+
+pytestmark = pytest.mark.gpu
+
+TOL_SCALE = 1e-6
+TOL_CODES = 1e-4
+TOL_OUT = 2e-3
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    from paper_2506_05413_b200 import build, binding as sr
+    build.build()
+    sr.load()
+    return torch, sr
+
+
+def _t(torch, a):
+    return torch.from_numpy(np.ascontiguousarray(a)).to("cuda:0")
+
+
+def _draw(seed, M, T, K1, I, N):
+    """A seeded block: Gaussian hidden states, Gaussian weights, and a few channels of the gated
+    product made massive (large rows of W_up and W_gate), as the paper describes the
+    down-projection's input."""
+    rng = np.random.default_rng(seed)
+    X = rng.standard_normal((M, K1)).astype(np.float16)
+    Xc = rng.standard_normal((T, K1)).astype(np.float16)
+    Wg = (rng.standard_normal((I, K1)) * 0.03).astype(np.float16)
+    Wu = (rng.standard_normal((I, K1)) * 0.03).astype(np.float16)
+    Wd = (rng.standard_normal((N, I)) * 0.02).astype(np.float16)
+    hot = rng.choice(I, size=3, replace=False)
+    Wu[hot] *= 30.0
+    Wg[hot] *= 4.0
+    d = np.where(rng.random(I) < 0.5, -1.0, 1.0).astype(np.float32)
+    if I == 14336:                       # 512 signs tiled 28 times, as for the down-projection workload
+        d = np.tile(d[:512], 28)
+    return X, Xc, Wg, Wu, Wd, d
+
+
+def _mismatch(got_packed, ref_packed):
+    a = orc.unpack_codes(got_packed).astype(np.int16)
+    b = orc.unpack_codes(ref_packed).astype(np.int16)
+    diff = np.abs(a - b)
+    return int(diff.max()), float((diff != 0).mean())
+
+
+def _rowwise_rel(got, want):
+    g, w = np.asarray(got, np.float64), np.asarray(want, np.float64)
+    den = np.abs(w).max(axis=1)
+    den = np.where(den == 0, 1.0, den)
+    return float((np.abs(g - w).max(axis=1) / den).max())
+
+
+def _run_block(torch, sr, X, Wg, Wu_abs, Wd, pre_w, d, clip_a=0.9, clip_w=1.0):
+    """The block on the device.  Returns device tensors of every stage."""
+    dev = "cuda:0"
+    M, K1 = X.shape
+    I, N = Wd.shape[1], Wd.shape[0]
+    f32 = lambda n: torch.empty(n, dtype=torch.float32, device=dev)
+    u8 = lambda r, c: torch.empty((r, c), dtype=torch.uint8, device=dev)
+    W_gu = _t(torch, np.concatenate([Wg, Wu_abs], axis=0))
+    wq_gu, dw_gu = u8(2 * I, K1 // 2), f32(2 * I)
+    sr.fuse_weights(W_gu, None, clip_w, wq_gu, dw_gu)
+    wq_d, dw_d = u8(N, I // 2), f32(N)
+    sr.fuse_weights(_t(torch, Wd), _t(torch, pre_w), clip_w, wq_d, dw_d)
+    xq, dx = u8(M, K1 // 2), f32(M)
+    sr.quant_act(_t(torch, X), None, clip_a, xq, dx)
+    Y_gu = torch.full((M, 2 * I), float("nan"), dtype=torch.float16, device=dev)
+    need = sr.workspace_bytes(M, 2 * I, K1)
+    sr.linear(xq, dx, wq_gu, dw_gu, Y_gu, torch.empty(need, dtype=torch.uint8, device=dev) if need else None)
+    hq, dh = u8(M, I // 2), f32(M)
+    # the two halves of the fused output, read in place (row stride 2 I)
+    sr.quant_act_glu(Y_gu[:, :I], Y_gu[:, I:], _t(torch, d), clip_a, hq, dh)
+    Y = torch.full((M, N), float("nan"), dtype=torch.float16, device=dev)
+    need = sr.workspace_bytes(M, N, I)
+    sr.linear(hq, dh, wq_d, dw_d, Y, torch.empty(need, dtype=torch.uint8, device=dev) if need else None)
+    torch.cuda.synchronize()
+    assert sr.device_status() == 0
+    return dict(wq_gu=wq_gu, dw_gu=dw_gu, wq_d=wq_d, dw_d=dw_d, xq=xq, dx=dx, Y_gu=Y_gu, hq=hq, dh=dh, Y=Y)
+
+
+def _check_rows(g, rows, X, Wg, Wu_abs, Wd, pre_w, d, w_rows_gu, w_rows_d):
+    """Staged comparison on the token rows `rows` (all output channels) and on sampled weight rows."""
+    K1 = X.shape[1]
+    I = Wd.shape[1]
+    cpu = {k: v.cpu().numpy() for k, v in g.items() if k not in ("Y_gu", "Y")}
+    Y_gu = g["Y_gu"].cpu().numpy()
+    Y = g["Y"].cpu().numpy()
+    # offline: sampled output channels of both weight matrices
+    W_gu = np.concatenate([Wg, Wu_abs], axis=0)
+    for W, pre, width, q, step, sel in ((W_gu, None, K1, cpu["wq_gu"], cpu["dw_gu"], w_rows_gu),
+                                        (Wd, pre_w, I, cpu["wq_d"], cpu["dw_d"], w_rows_d)):
+        q_ref, step_ref, _ = orc.fuse_weights(W[sel], pre, width, 1.0)
+        assert np.abs(step[sel] / step_ref - 1).max() <= TOL_SCALE
+        worst, frac = _mismatch(q[sel], q_ref)
+        assert worst <= 1 and frac <= TOL_CODES
+    # online stage 1: the block input
+    q_ref, step_ref, _ = orc.quant_act(X[rows], None, K1, 0.9)
+    assert np.abs(cpu["dx"][rows] / step_ref - 1).max() <= TOL_SCALE
+    worst, frac = _mismatch(cpu["xq"][rows], q_ref)
+    assert worst <= 1 and frac <= max(TOL_CODES, 1.5 / (2 * q_ref.size))
+    # gate/up layer on the GPU's codes: both halves of the fused output
+    Ygu_ref = orc.linear(cpu["xq"][rows], cpu["dx"][rows], cpu["wq_gu"], cpu["dw_gu"])
+    assert _rowwise_rel(Y_gu[rows][:, :I], Ygu_ref[:, :I]) <= TOL_OUT
+    assert _rowwise_rel(Y_gu[rows][:, I:], Ygu_ref[:, I:]) <= TOL_OUT
+    # the online edge of Fig. 2 on the GPU's fp16 gate/up outputs
+    hq_ref, dh_ref, _ = orc.quant_act_glu(Y_gu[rows][:, :I], Y_gu[rows][:, I:], d, I, 0.9)
+    assert np.abs(cpu["dh"][rows] / dh_ref - 1).max() <= TOL_SCALE
+    worst, frac = _mismatch(cpu["hq"][rows], hq_ref)
+    assert worst <= 1 and frac <= max(TOL_CODES, 1.5 / (2 * hq_ref.size))
+    # down layer on the GPU's codes
+    Y_ref = orc.linear(cpu["hq"][rows], cpu["dh"][rows], cpu["wq_d"], cpu["dw_d"])
+    assert _rowwise_rel(Y[rows], Y_ref) <= TOL_OUT
+    return Y
+
+
+@pytest.mark.parametrize("M,K1,I,N", [(24, 128, 512, 64), (70, 512, 28 * 16, 136), (300, 256, 4096, 264)])
+def test_ffn_block_reduced_sizes_in_full(env, M, K1, I, N):
+    torch, sr = env
+    X, Xc, Wg, Wu, Wd, d = _draw(M + I, M, 64, K1, I, N)
+    _, _, s = orc.ffn_calibrate(Xc, Wg, Wu, Wd, 0.5)
+    Wu_abs = orc.absorb_into_up(Wu, s).astype(np.float16)
+    pre_w = (s.astype(np.float64) * d).astype(np.float32)
+    g = _run_block(torch, sr, X, Wg, Wu_abs, Wd, pre_w, d)
+    rows = np.arange(M)
+    Y = _check_rows(g, rows, X, Wg, Wu_abs, Wd, pre_w, d, np.arange(2 * I), np.arange(N))
+    # the whole chain against the oracle's own chain: close, though not staged (ties upstream move codes)
+    ref = orc.ffn_block(X, Wg, Wu, Wd, s, d)
+    assert np.array_equal(ref["W_up_abs"], Wu_abs)
+    want = ref["Y"].astype(np.float64)
+    assert np.linalg.norm(Y.astype(np.float64) - want) <= 0.05 * np.linalg.norm(want)
+    # and the block still computes the unquantized function (4-bit accuracy)
+    plain = orc.ffn_plain_fp64(X, Wg, Wu, Wd)
+    assert np.linalg.norm(Y.astype(np.float64) - plain) <= 0.5 * np.linalg.norm(plain)
+
+
+def test_ffn_block_model_widths_sampled_rows(env):
+    """4096 -> 2 x 14336 -> 4096 (the gate/up and down shapes of the workloads), 512 tokens: the
+    two-CTA tcgen05 kernel serves both layers and the K = 14336 kernel the online edge; the oracle
+    follows 24 sampled tokens through every stage and 32 sampled output channels of each weight."""
+    torch, sr = env
+    M, K1, I, N = 512, 4096, 14336, 4096
+    X, Xc, Wg, Wu, Wd, d = _draw(11, M, 128, K1, I, N)
+    _, _, s = orc.ffn_calibrate(Xc, Wg, Wu, Wd, 0.5)
+    Wu_abs = orc.absorb_into_up(Wu, s).astype(np.float16)
+    pre_w = (s.astype(np.float64) * d).astype(np.float32)
+    g = _run_block(torch, sr, X, Wg, Wu_abs, Wd, pre_w, d)
+    rng = np.random.default_rng(12)
+    rows = np.sort(np.concatenate([[0, 127, 128, 255, 256, M - 1], rng.choice(np.arange(1, M - 1), 18, replace=False)]))
+    rows = np.unique(rows)
+    w_gu = np.unique(np.concatenate([[0, I - 1, I, 2 * I - 1], rng.choice(2 * I, 28, replace=False)]))
+    w_d = np.unique(np.concatenate([[0, N - 1], rng.choice(N, 30, replace=False)]))
+    _check_rows(g, rows, X, Wg, Wu_abs, Wd, pre_w, d, w_gu, w_d)
+    assert bool(torch.isfinite(g["Y"]).all()) and bool(torch.isfinite(g["Y_gu"]).all())
