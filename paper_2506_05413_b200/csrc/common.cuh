@@ -57,6 +57,28 @@ inline int device_sm_count() {
   return n;
 }
 
+// cuTensorMapEncodeTiled, looked up through the runtime (the library does not link libcuda).
+#ifdef CUDA_VERSION
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                      const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                      CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline TensorMapEncodeFn tensor_map_encoder() {
+  static std::atomic<TensorMapEncodeFn> cached{nullptr};
+  TensorMapEncodeFn fn = cached.load(std::memory_order_acquire);
+  if (fn == nullptr) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess) {
+      fn = reinterpret_cast<TensorMapEncodeFn>(ptr);
+      cached.store(fn, std::memory_order_release);
+    }
+  }
+  return fn;
+}
+#endif
+
 inline int launch_status() {
   return cudaGetLastError() == cudaSuccess ? SMOOTHROT_OK : SMOOTHROT_CUDA_ERROR;
 }

@@ -130,7 +130,7 @@ def _check_rows(g, rows, X, Wg, Wu_abs, Wd, pre_w, d, w_rows_gu, w_rows_d):
     return Y
 
 
-@pytest.mark.parametrize("M,K1,I,N", [(24, 128, 512, 64), (70, 512, 28 * 16, 136), (300, 256, 4096, 264)])
+@pytest.mark.parametrize("M,K1,I,N", [(24, 128, 512, 64), (70, 512, 28 * 32, 136), (300, 256, 4096, 264)])
 def test_ffn_block_reduced_sizes_in_full(env, M, K1, I, N):
     torch, sr = env
     X, Xc, Wg, Wu, Wd, d = _draw(M + I, M, 64, K1, I, N)
