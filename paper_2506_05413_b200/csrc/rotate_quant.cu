@@ -14,6 +14,8 @@
 //                           shared-memory transpose, codes assembled with warp
 //                           shuffles so that every global access is coalesced.
 //   paley512_kernel         K = 14336 = 28 x 512: see below.
+#include <cuda.h>
+
 #include <type_traits>
 
 #include "common.cuh"
@@ -249,6 +251,8 @@ constexpr unsigned long long kLoadWaitLimitNs = 2000000000ull;  // 2 s
 
 // Set when a bounded wait for a row copy ran out (read by smoothrot_device_status).
 __device__ int g_rotate_status = 0;
+// Limit of the bounded waits of the row kernels in nanoseconds (a test shortens it).
+__device__ unsigned long long g_rotate_wait_limit_ns = kLoadWaitLimitNs;
 
 __device__ __forceinline__ void group_barrier(int group) {
   asm volatile("bar.sync %0, 64;" ::"r"(group + 1) : "memory");
@@ -276,7 +280,7 @@ __device__ __forceinline__ bool wait_row_copy(uint32_t bar, uint32_t parity) {
     if ((spin & 255u) == 0u) {
       unsigned long long now;
       asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
-      if (now - t0 > kLoadWaitLimitNs) {
+      if (now - t0 > g_rotate_wait_limit_ns) {
         atomicCAS(&g_rotate_status, 0, 16);
         return false;
       }
@@ -537,6 +541,10 @@ walsh4096_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
   }
   }  // rows of this group
 }
+
+}  // namespace smoothrot
+#include "walsh4096_tc.cuh"
+namespace smoothrot {
 
 // ---------------------------------------------------------------------------
 // K = 14336 = 28 x 512  (index j = a * 512 + b; H = kron(H28, H512)).
@@ -924,6 +932,42 @@ static int launch_rotate(const void* X, int64_t rows, int64_t K, int64_t ld, con
   }
   const __half* x = static_cast<const __half*>(X);
   const __half* u = static_cast<const __half*>(U);
+  if (K == 4096 && !glu && pre == nullptr && rows >= 512) {
+    // No diagonal: the order-128 factor of the rotation on the tensor cores (walsh4096_tc.cuh).
+    // A few hundred rows or fewer finish sooner in the register kernel below (shorter set-up).
+    const bool low = kQuant && (7.0f / clip >= 8.49f);
+    // the rows as a [rows][32 groups][2 halves][64 values] tensor; a box = one K half of 8 rows
+    CUtensorMap xmap;
+    TensorMapEncodeFn encode = tensor_map_encoder();
+    if (encode == nullptr) return SMOOTHROT_CUDA_ERROR;
+    const cuuint64_t dims[4] = {64, 2, 32, cuuint64_t(rows)};
+    const cuuint64_t strides[3] = {128, 256, cuuint64_t(ld) * sizeof(__half)};
+    const int sms = device_sm_count();
+    // batches of six rows for long inputs, of four (finer granularity, shorter tail) otherwise
+    const bool six = rows >= int64_t(48) * sms;
+    const int tokens = six ? 6 : 4;
+    const cuuint32_t box[4] = {64, 1, 32, cuuint32_t(tokens)};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    if (encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<__half*>(x), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return SMOOTHROT_CUDA_ERROR;
+    const int64_t batches = (rows + tokens - 1) / tokens;
+    const unsigned grid = unsigned(batches < sms ? batches : sms);
+    if (six) {
+      auto kern = low ? wtc::walsh4096_tc_kernel<kQuant, true, 6> : wtc::walsh4096_tc_kernel<kQuant, false, 6>;
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, wtc::Cfg<6>::kSmemBytes) != cudaSuccess)
+        return SMOOTHROT_CUDA_ERROR;
+      kern<<<grid, wtc::Cfg<6>::kThreads, wtc::Cfg<6>::kSmemBytes, stream>>>(xmap, rows, clip, q_out, step_out, y_out);
+    } else {
+      auto kern = low ? wtc::walsh4096_tc_kernel<kQuant, true, 4> : wtc::walsh4096_tc_kernel<kQuant, false, 4>;
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, wtc::Cfg<4>::kSmemBytes) != cudaSuccess)
+        return SMOOTHROT_CUDA_ERROR;
+      kern<<<grid, wtc::Cfg<4>::kThreads, wtc::Cfg<4>::kSmemBytes, stream>>>(xmap, rows, clip, q_out, step_out, y_out);
+    }
+    count_launch();
+    return launch_status();
+  }
   if (K == 4096 && !glu) {
     // codes below -8 can only come up when the row maximum sits at 8.5 steps or more
     const bool low = kQuant && (7.0f / clip >= 8.49f);
