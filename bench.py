@@ -2,6 +2,7 @@
 """Benchmark of the SmoothRot W4A4 linear layer on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3] [--per-config 0|1]
+    python bench.py --workload cfg4 --shape gate_up --tokens 1 ...   # one point of the token-count sweep
     python bench.py --impl reference ...        # the CPU oracle on the host cores
 
 One "step" is one pass of the whole path over one batch of seeded synthetic
@@ -251,7 +252,8 @@ class DeviceSet:
         self.amax, self.s, self.pre_w, self.pre_x = f32(K), f32(K), f32(K), f32(K)
         self.wq = torch.empty((N, K // 2), dtype=torch.uint8, device=dev)
         self.xq = torch.empty((M, K // 2), dtype=torch.uint8, device=dev)
-        self.dw, self.dx = f32(N), f32(M)
+        self.xq2 = torch.empty((M, K // 2), dtype=torch.uint8, device=dev)   # outputs of the call without a diagonal
+        self.dw, self.dx, self.dx2 = f32(N), f32(M), f32(M)
         self.Y = torch.empty((M, N), dtype=torch.float16, device=dev)
         need = sr.workspace_bytes(M, N, K)
         self.ws = torch.empty(need, dtype=torch.uint8, device=dev) if need else None
@@ -279,13 +281,17 @@ def step_calls(sr, case, ds):
         "fuse_weights": lambda: sr.fuse_weights(ds.W, ds.pre_w, case.clip_w, ds.wq, ds.dw),
         "quant_act": lambda: sr.quant_act(ds.X, ds.pre_x, case.clip_a, ds.xq, ds.dx),
         "linear": lambda: sr.linear(ds.xq, ds.dx, ds.wq, ds.dw, ds.Y, ds.ws),
+        # not a step of the path: the exact online Hadamard of the paper's deployment (Lambda^-1 absorbed
+        # by the producing layer, no sign diagonal), timed beside quant_act for comparison
+        "quant_act_exact": lambda: sr.quant_act(ds.X, None, case.clip_a, ds.xq2, ds.dx2),
     }
 
 
 def gpu_step(sr, case, ds):
     """The whole path on one buffer set, call by call (eager launches)."""
-    for fn in step_calls(sr, case, ds).values():
-        fn()
+    calls = step_calls(sr, case, ds)
+    for name in CALLS:
+        calls[name]()
 
 
 def max_over_ranks(torch, dist, value, dev):
@@ -415,6 +421,11 @@ def measure_layer(torch, sr, case, dev, rec, local, min_seconds, sampler_on=True
             entry["TOPS"] = tops
             entry["frac"] = linear_fracs(tops, rec)
         out[name] = entry
+    exact = [capture(torch, [step_calls(sr, case, ds)["quant_act_exact"]]) for ds in sets]
+    mean, best, regions = time_replays(torch, exact, min_seconds)
+    out["quant_act_exact"] = {"us": mean * 1e6, "us_min": best * 1e6, "GB/s": abytes["quant_act"] / mean / 1e9,
+                              "frac_hbm": abytes["quant_act"] / mean / 1e9 / rec["hbm_gbs"],
+                              "note": "smoothrot_quant_act without a diagonal (exact online Hadamard); not part of the step"}
     mean, best, regions = time_replays(torch, whole, min_seconds)
     out["step"] = {"us": mean * 1e6, "us_min": best * 1e6, "TOPS": layer_ops(M, N, K) / mean / 1e12}
     out["clocks"] = sampler.stop()
@@ -454,6 +465,8 @@ def measure_sweep(torch, sr, dev, rec, local, min_seconds, sampler_on=True):
             torch.cuda.synchronize()
             gq = [capture(torch, [lambda s=s: sr.quant_act(s[0], full.pre_x, case.clip_a, s[1], s[2])]) for s in sets]
             gl = [capture(torch, [lambda s=s: sr.linear(s[1], s[2], s[3], s[4], s[5], s[6])]) for s in sets]
+            ge = [capture(torch, [lambda s=s: sr.quant_act(s[0], None, case.clip_a, s[1], s[2])]) for s in sets]
+            te, te_min, _ = time_replays(torch, ge, min_seconds)
             tq, tq_min, _ = time_replays(torch, gq, min_seconds)
             tl, tl_min, _ = time_replays(torch, gl, min_seconds)
             ops = layer_ops(M, N, K)
@@ -461,6 +474,7 @@ def measure_sweep(torch, sr, dev, rec, local, min_seconds, sampler_on=True):
                    "linear_kernel": sr.linear_plan_name(M, N, K),
                    "quant_act_us": tq * 1e6, "quant_act_us_min": tq_min * 1e6,
                    "quant_act_GBs": (2.5 * M * K + 4 * M + 4 * K) / tq / 1e9,
+                   "quant_act_exact_us": te * 1e6, "quant_act_exact_GBs": (2.5 * M * K + 4 * M) / te / 1e9,
                    "linear_us": tl * 1e6, "linear_us_min": tl_min * 1e6, "linear_TOPS": ops / tl / 1e12,
                    "linear_frac_bf16_burst_x2": ops / tl / 1e12 / rec["int8_from_bf16_burst"],
                    "weight_stream_GBs": 0.5 * N * K / tl / 1e9,
@@ -468,7 +482,7 @@ def measure_sweep(torch, sr, dev, rec, local, min_seconds, sampler_on=True):
                    "algorithmic": {"ops": ops, "linear_bytes": 0.5 * M * K + 0.5 * N * K + 2.0 * M * N + 4.0 * (M + N),
                                    "quant_act_bytes": 2.5 * M * K + 4 * M + 4 * K}}
             shape_rows.append(row)
-            del sets, gq, gl
+            del sets, gq, gl, ge
             torch.cuda.empty_cache()
         clocks = sampler.stop()
         for row in shape_rows:
@@ -583,6 +597,11 @@ def run_gpu(args, case, desc):
     for name in CALLS:
         mean, best, _ = time_replays(torch, single[name], 0.25 if name == "linear" else 0.1)
         call_ms[name], call_ms_min[name] = mean * 1e3, best * 1e3
+    for ds in sets:
+        step_calls(sr, case, ds)["quant_act_exact"]()
+    torch.cuda.synchronize()
+    exact_graphs = [capture(torch, [step_calls(sr, case, ds)["quant_act_exact"]]) for ds in sets]
+    exact_mean, exact_min, _ = time_replays(torch, exact_graphs, 0.1)
     clocks_calls = sampler2.stop() if rank == 0 else None
     call_ms_alone_linear = call_ms["linear"]
     call_ms["linear"] = linear_live_ms
@@ -674,6 +693,12 @@ def run_gpu(args, case, desc):
     per_call["linear"]["TOPS"] = ops / (call_ms["linear"] * 1e-3) / 1e12
     per_call["linear"]["frac_int8_peak"] = per_call["linear"]["TOPS"] / int8_peak
     per_call["linear"]["ms_alone"] = call_ms_alone_linear
+    per_call["quant_act_exact"] = {
+        "ms": exact_mean * 1e3, "ms_min_alone": exact_min * 1e3, "GB/s": abytes["quant_act"] / exact_mean / 1e9,
+        "frac_hbm": abytes["quant_act"] / exact_mean / 1e9 / peaks["hbm_gbs"],
+        "frac_hbm_nominal_8000": abytes["quant_act"] / exact_mean / 1e9 / NOMINAL_HBM_GBS,
+        "note": "smoothrot_quant_act without a diagonal (the exact online Hadamard of the paper's deployment, "
+                "Lambda^-1 absorbed by the producing layer); timed alone, not part of the step"}
     per_call["clocks"] = clocks_calls
 
     # ---- the other workloads, one GPU only (each with its own clock record) ----
@@ -739,14 +764,21 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
-    ap.add_argument("--workload", choices=sorted(WORKLOADS), default="cfg3")
+    ap.add_argument("--workload", choices=sorted(WORKLOADS) + ["cfg4"], default="cfg3")
+    ap.add_argument("--shape", choices=[n for n, _, _ in synth.BLOCK_SHAPES], default="gate_up",
+                    help="with --workload cfg4: the linear shape of the decoder block")
+    ap.add_argument("--tokens", type=int, default=1, help="with --workload cfg4: the token count M")
     ap.add_argument("--per-config", type=int, default=1, help="0: skip the records of the other workloads")
     ap.add_argument("--min-region-s", type=float, default=0.5,
                     help="device seconds the repeated K-step regions must cover")
     ap.add_argument("--min-config-s", type=float, default=0.06,
                     help="device seconds per timed call in the per-config records")
     args = ap.parse_args()
-    maker, desc = WORKLOADS[args.workload]
+    if args.workload == "cfg4":
+        maker = lambda: synth.config4(args.shape, args.tokens)
+        desc = f"configs[4]: one point of the token-count sweep, shape {args.shape}, M = {args.tokens}"
+    else:
+        maker, desc = WORKLOADS[args.workload]
     rank = int(os.environ.get("RANK", "0"))
     if args.impl == "reference":
         if rank != 0:

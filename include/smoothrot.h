@@ -214,8 +214,8 @@ int smoothrot_linear(const uint8_t* Xq, const float* dx, int64_t M,
  * many bytes occupied until the process exits, whether or not this entry
  * point is ever called there.
  *
- * Same arguments, results and error behaviour as smoothrot_linear, minus the
- * workspace pair.  The call itself allocates and frees nothing.  Shapes whose
+ * Same arguments, results and error behaviour as smoothrot_linear (the same
+ * checks in the same order, before anything else), minus the workspace pair.  The call itself allocates and frees nothing.  Shapes whose
  * smoothrot_workspace_bytes(M, N, K) exceeds SMOOTHROT_STATIC_SCRATCH_BYTES
  * are refused with SMOOTHROT_STATIC_SCRATCH_EXCEEDED and nothing is enqueued
  * (use smoothrot_linear with your own workspace for those).
@@ -309,6 +309,20 @@ int smoothrot_debug_hadamard_heads(const void* X_f16, int64_t M, int64_t n_heads
 int smoothrot_debug_gemm_i32(const uint8_t* Xq, int64_t M, const uint8_t* Wq, int64_t N,
                              int64_t K, int32_t* acc,
                              void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Test exports for the bounded device-side waits (no passage of the paper: the kernels never
+ * spin without bound, and these two calls let a test see a wait run out without hanging
+ * anything).
+ *   smoothrot_debug_set_wait_limit_ns: host, synchronous.  Sets the limit of every bounded wait
+ *     of the library's kernels on the current device, in nanoseconds; 0 restores the default
+ *     (two seconds).
+ *   smoothrot_debug_wait_expiry: enqueues one warp that waits, through the same bounded wait as
+ *     the GEMM kernels, on a barrier nobody arrives on.  When the limit has passed the warp
+ *     records code 7 in the status word smoothrot_device_status reads, and the kernel returns.
+ */
+int smoothrot_debug_set_wait_limit_ns(uint64_t ns);
+int smoothrot_debug_wait_expiry(void* stream);
 
 /* Host. Writes the library's own order-28 Paley matrix, row-major, entries
  * +1 / -1, into out[784] (a host buffer). */

@@ -40,6 +40,8 @@ SIGNATURES = {
     "smoothrot_debug_hadamard": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp]),
     "smoothrot_debug_hadamard_heads": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _vp, _vp]),
     "smoothrot_debug_gemm_i32": (_int, [_vp, _i64, _vp, _i64, _i64, _vp, _vp, _sz, _vp]),
+    "smoothrot_debug_set_wait_limit_ns": (_int, [ctypes.c_uint64]),
+    "smoothrot_debug_wait_expiry": (_int, [_vp]),
     "smoothrot_paley28": (_int, [_vp]),
     "smoothrot_device_status": (_int, [ctypes.POINTER(_int), _int]),
     "smoothrot_launch_count": (_i64, []),
@@ -351,6 +353,16 @@ def paley28():
     buf = (ctypes.c_int8 * 784)()
     _check(load().smoothrot_paley28(ctypes.cast(buf, ctypes.c_void_p)))
     return [[int(buf[r * 28 + c]) for c in range(28)] for r in range(28)]
+
+
+def debug_set_wait_limit_ns(ns: int) -> None:
+    """Limit of the kernels' bounded waits on the current device (0: back to two seconds)."""
+    _check(load().smoothrot_debug_set_wait_limit_ns(int(ns)))
+
+
+def debug_wait_expiry() -> None:
+    """Enqueues the probe whose bounded wait is certain to run out (it returns normally)."""
+    _check(load().smoothrot_debug_wait_expiry(_stream()))
 
 
 def device_status(clear: bool = True) -> int:

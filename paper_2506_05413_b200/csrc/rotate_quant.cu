@@ -1058,6 +1058,14 @@ int smoothrot_rotate_status_word(int* value, int clear) {
   return SMOOTHROT_OK;
 }
 
+// Host. Limit of the bounded waits of the row transform kernels on the current device
+// (0 restores the default of two seconds).
+int smoothrot_rotate_set_wait_limit_ns(uint64_t ns) {
+  const unsigned long long v = ns == 0 ? smoothrot::kLoadWaitLimitNs : static_cast<unsigned long long>(ns);
+  if (cudaMemcpyToSymbol(smoothrot::g_rotate_wait_limit_ns, &v, sizeof(v)) != cudaSuccess) return SMOOTHROT_CUDA_ERROR;
+  return SMOOTHROT_OK;
+}
+
 int smoothrot_paley28(int8_t* out_host) {
   if (out_host == nullptr) return SMOOTHROT_INVALID_ARG;
   for (int r = 0; r < 28; ++r)

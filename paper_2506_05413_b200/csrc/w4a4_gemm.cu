@@ -41,6 +41,8 @@
 
 // defined with the row transform kernels: their timeout word
 extern "C" int smoothrot_rotate_status_word(int* value, int clear);
+// defined with the row transform kernels: the limit of their bounded waits
+extern "C" int smoothrot_rotate_set_wait_limit_ns(uint64_t ns);
 
 namespace smoothrot {
 namespace gemm {
@@ -52,11 +54,14 @@ constexpr int kWidenWarps = 8;
 constexpr int kEpiWarps = 4;
 constexpr int kThreads = 32 * (2 + kWidenWarps + kEpiWarps);
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
+constexpr unsigned long long kDrainNs = 50000ull;           // pause before leaving after a timeout
 
 __device__ int g_device_status = 0;
+// Limit of every bounded wait of these kernels, in nanoseconds (a test shortens it).
+__device__ unsigned long long g_wait_limit_ns = kWaitLimitNs;
 
 enum TimeoutSite { kSiteProducer = 1, kSiteWidenFull = 2, kSiteWidenEmpty = 3, kSiteMmaAcc = 4,
-                   kSiteMmaWide = 5, kSiteEpilogue = 6 };
+                   kSiteMmaWide = 5, kSiteEpilogue = 6, kSiteProbe = 7 };
 
 template <int BN>
 struct Tile {
@@ -107,7 +112,8 @@ __device__ __forceinline__ unsigned long long global_ns() {
   return t;
 }
 
-// Waits for the barrier phase with the given parity, at most kWaitLimitNs.
+// Waits for the barrier phase with the given parity, at most g_wait_limit_ns (2 s unless a test
+// has shortened it).
 // Returns false if the wait ran out or another role of this CTA gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int site) {
   if (mbar_try_wait(bar, parity)) return true;
@@ -116,13 +122,22 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try_wait(bar, parity)) return true;
     if ((spin & 63u) == 0u) {
       if (*abort_flag != 0) return false;
-      if (global_ns() - t0 > kWaitLimitNs) {
+      if (global_ns() - t0 > g_wait_limit_ns) {
         *abort_flag = 1;
         atomicCAS(&g_device_status, 0, site);
         return false;
       }
     }
   }
+}
+
+// Wind-down after a timeout: copies and tensor-core operations this CTA started may still be on
+// their way into its shared and tensor memory.  Every thread pauses long enough for them to land
+// (they complete in microseconds once issued) before the CTA gives its memory back.
+__device__ __forceinline__ void drain_after_abort(volatile int* abort_flag) {
+  if (*abort_flag == 0) return;
+  const unsigned long long t0 = global_ns();
+  while (global_ns() - t0 < kDrainNs) __nanosleep(1000);
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
@@ -440,6 +455,7 @@ w4a4_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     }
   }
 
+  drain_after_abort(abort_flag);
   tcgen05_fence_before();
   __syncthreads();
   if (warp == 1) {
@@ -909,6 +925,7 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
     if (lane == 0) tma_store_wait_all();
   }
 
+  drain_after_abort(abort_flag);
   tcgen05_fence_before();
   __syncthreads();
   cluster_sync_all();  // both CTAs are done with both halves of tensor memory
@@ -1179,6 +1196,7 @@ w4a4_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     }
   }
 
+  drain_after_abort(abort_flag);
   tcgen05_fence_before();
   __syncthreads();
   if (p.cluster_reduce) {
@@ -1450,6 +1468,24 @@ static int launch_decode(const uint8_t* Xq, const uint8_t* Wq, int M, int N, int
   return launch_status();
 }
 
+// Test probe: one warp waits, through the same bounded wait as the kernels above, on an mbarrier
+// that nobody ever arrives on.  The wait runs out after g_wait_limit_ns, records kSiteProbe in the
+// status word and the kernel returns normally.
+__global__ void wait_expiry_probe_kernel() {
+  __shared__ __align__(8) unsigned long long bar_storage;
+  __shared__ int abort_word;
+  const uint32_t bar = smem_u32(&bar_storage);
+  if (threadIdx.x == 0) {
+    abort_word = 0;
+    mbar_init(bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  volatile int* abort_flag = &abort_word;
+  (void)mbar_wait(bar, 0u, abort_flag, kSiteProbe);
+  drain_after_abort(abort_flag);
+}
+
 // ---------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------
@@ -1462,17 +1498,17 @@ struct Plan {
   int splits;
 };
 
+// Number of SMs of the current device, remembered per device.
 static int sm_count() {
-  static int cached = 0;
-  if (cached == 0) {
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess &&
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
-      cached = n;
-    else
-      return 148;
-  }
-  return cached;
+  constexpr int kSlots = 64;
+  static std::atomic<int> cached[kSlots];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kSlots) return 148;
+  int n = cached[dev].load(std::memory_order_relaxed);
+  if (n > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+  cached[dev].store(n, std::memory_order_relaxed);
+  return n;
 }
 
 constexpr int kPairSplitMinBlocks = 32;   // k-blocks per split below which the extra pass over the partial sums costs more than it saves
@@ -1573,11 +1609,24 @@ static bool make_map_y(CUtensorMap* map, __half* Y, int64_t M, int64_t N, int64_
          CUDA_SUCCESS;
 }
 
+// Raises a kernel's dynamic shared-memory limit; once per kernel, device and process.  kTag tells
+// the kernels apart (several share one function type, so the type alone would not).
+template <int kTag, typename Kern>
+static bool allow_smem(Kern kern, int bytes) {
+  constexpr int kSlots = 64;
+  static std::atomic<int> done[kSlots];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kSlots) dev = kSlots - 1;
+  if (done[dev].load(std::memory_order_acquire) >= bytes) return true;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+  done[dev].store(bytes, std::memory_order_release);
+  return true;
+}
+
 template <int BN>
 static int launch_stream(const CUtensorMap& ma, const CUtensorMap& mb, const Params& p, cudaStream_t st) {
   auto kern = w4a4_gemm_stream_kernel<BN>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Stream<BN>::kSmemBytes) != cudaSuccess)
-    return SMOOTHROT_CUDA_ERROR;
+  if (!allow_smem<1000 + BN>(kern, Stream<BN>::kSmemBytes)) return SMOOTHROT_CUDA_ERROR;
   const int total = p.tiles_a * p.tiles_b * p.splits;   // one CTA per (channel tile, token tile, k-split)
   if (p.cluster_reduce) {
     cudaLaunchConfig_t cfg{};
@@ -1607,8 +1656,7 @@ static int launch_stream(const CUtensorMap& ma, const CUtensorMap& mb, const Par
 template <int BN>
 static int launch_tile(const CUtensorMap& ma, const CUtensorMap& mb, const Params& p, cudaStream_t st) {
   auto kern = w4a4_gemm_kernel<BN>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Tile<BN>::kSmemBytes) != cudaSuccess)
-    return SMOOTHROT_CUDA_ERROR;
+  if (!allow_smem<2000 + BN>(kern, Tile<BN>::kSmemBytes)) return SMOOTHROT_CUDA_ERROR;
   const int total = p.tiles_a * p.tiles_b * p.splits;
   const int grid = total < sm_count() ? total : sm_count();
   kern<<<grid, kThreads, Tile<BN>::kSmemBytes, st>>>(ma, mb, p);
@@ -1626,13 +1674,18 @@ static int launch_splitk_reduce(const void* workspace, int splits, int64_t M, in
   return launch_status();
 }
 
-static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq, const float* dw, int64_t N,
-               int64_t K, __half* Y, int64_t ldy, int32_t* acc_out, void* workspace, size_t workspace_bytes,
-               cudaStream_t st) {
+// Argument checks shared by every entry point of the layer.  Returns SMOOTHROT_OK with *empty set
+// when there is nothing to compute.
+static int check_args(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq, const float* dw, int64_t N,
+                      int64_t K, const __half* Y, int64_t ldy, const int32_t* acc_out, bool* empty) {
+  *empty = false;
   if (M < 0 || N < 0 || K <= 0) return SMOOTHROT_INVALID_ARG;
   if (K % kWideRow != 0 || K > 65536) return SMOOTHROT_UNSUPPORTED_K;
   if (N % 8 != 0) return SMOOTHROT_INVALID_ARG;
-  if (M == 0 || N == 0) return SMOOTHROT_OK;
+  if (M == 0 || N == 0) {
+    *empty = true;
+    return SMOOTHROT_OK;
+  }
   if (M > 0x7fffffffLL / 2 || N > 0x7fffffffLL / 2) return SMOOTHROT_INVALID_ARG;
   if (Xq == nullptr || Wq == nullptr) return SMOOTHROT_INVALID_ARG;
   if (!aligned16(Xq) || !aligned16(Wq)) return SMOOTHROT_BAD_ALIGNMENT;
@@ -1643,6 +1696,15 @@ static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq,
     if (acc_out == nullptr) return SMOOTHROT_INVALID_ARG;
     if (!aligned16(acc_out)) return SMOOTHROT_BAD_ALIGNMENT;
   }
+  return SMOOTHROT_OK;
+}
+
+static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq, const float* dw, int64_t N,
+               int64_t K, __half* Y, int64_t ldy, int32_t* acc_out, void* workspace, size_t workspace_bytes,
+               cudaStream_t st) {
+  bool empty = false;
+  const int args_rc = check_args(Xq, dx, M, Wq, dw, N, K, Y, ldy, acc_out, &empty);
+  if (args_rc != SMOOTHROT_OK || empty) return args_rc;
   Plan pl = make_plan(M, N, K);
   size_t need = (pl.splits > 1 && !pl.cluster) ? size_t(pl.splits) * size_t(M) * size_t(N) * sizeof(int32_t) : 0;
   if (pl.pair && need > 0 && (workspace == nullptr || workspace_bytes < need)) {
@@ -1698,8 +1760,7 @@ static int run(const uint8_t* Xq, const float* dx, int64_t M, const uint8_t* Wq,
     CUtensorMap my = ma;   // only read by the kernel when Y is written
     if (p.Y != nullptr && !make_map_y(&my, p.Y, M, N, ldy)) return SMOOTHROT_CUDA_ERROR;
     auto kern = w4a4_gemm_pair_tmem_kernel;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PairT::kSmemBytes) != cudaSuccess)
-      return SMOOTHROT_CUDA_ERROR;
+    if (!allow_smem<3000>(kern, PairT::kSmemBytes)) return SMOOTHROT_CUDA_ERROR;
     const int total = p.tiles_a * p.tiles_b * pl.splits;
     const int pairs = sm_count() / 2;
     const int grid = 2 * (total < pairs ? total : pairs);
@@ -1763,6 +1824,11 @@ int smoothrot_linear_static_scratch(const uint8_t* Xq, const float* dx, int64_t 
                                     void* stream) {
   using namespace smoothrot::gemm;
   if (M > 0 && N > 0 && Y_f16 == nullptr) return SMOOTHROT_INVALID_ARG;
+  // the same argument checks, in the same order, as smoothrot_linear: only a valid call can be
+  // refused for its size
+  bool empty = false;
+  const int args_rc = check_args(Xq, dx, M, Wq, dw, N, K, static_cast<const __half*>(Y_f16), ldy, nullptr, &empty);
+  if (args_rc != SMOOTHROT_OK || empty) return args_rc;
   size_t need = smoothrot_workspace_bytes(M, N, K);
   if (need > kStaticScratchBytes) {
     // prefill shapes split K only as an optimisation and run without scratch memory as well
@@ -1779,6 +1845,18 @@ int smoothrot_linear_static_scratch(const uint8_t* Xq, const float* dx, int64_t 
   // and nothing has to be cleared.
   return run(Xq, dx, M, Wq, dw, N, K, static_cast<__half*>(Y_f16), ldy, nullptr, scratch,
              need > 0 ? kStaticScratchBytes : 0, static_cast<cudaStream_t>(stream));
+}
+
+int smoothrot_debug_set_wait_limit_ns(uint64_t ns) {
+  const unsigned long long v = ns == 0 ? smoothrot::gemm::kWaitLimitNs : static_cast<unsigned long long>(ns);
+  if (cudaMemcpyToSymbol(smoothrot::gemm::g_wait_limit_ns, &v, sizeof(v)) != cudaSuccess) return SMOOTHROT_CUDA_ERROR;
+  return smoothrot_rotate_set_wait_limit_ns(ns);
+}
+
+int smoothrot_debug_wait_expiry(void* stream) {
+  smoothrot::gemm::wait_expiry_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>();
+  smoothrot::count_launch();
+  return smoothrot::launch_status();
 }
 
 const char* smoothrot_linear_plan_name(int64_t M, int64_t N, int64_t K) {

@@ -345,6 +345,16 @@ walsh4096_tc_kernel(const __grid_constant__ CUtensorMap xmap, int64_t M, float c
     }
   }
 
+  if (*abort_flag != 0) {
+    // after a timeout: give copies and tensor-core operations already started the time to land
+    // before the CTA returns its shared and tensor memory
+    unsigned long long t0, now;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    do {
+      __nanosleep(1000);
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+    } while (now - t0 < 50000ull);
+  }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (warp == 1) {

@@ -327,10 +327,10 @@ def test_glu_quantized_codes_match_oracle(gu, K, M, use_pre):
     torch.cuda.synchronize()
     assert sr.device_status() == 0
     q_ref, step_ref, _ = orc.quant_act_glu(gate, up, pre, K, 0.9)
-    # the kernel evaluates the SiLU in fp32 with fast exp / divide: 1e-6 on the largest entry of a row
-    assert np.abs(step.cpu().numpy() / step_ref - 1).max() <= 2e-6
+    # the kernel evaluates the SiLU in fp32 (library exponential, IEEE division): the stated budgets hold
+    assert np.abs(step.cpu().numpy() / step_ref - 1).max() <= TOL_SCALE
     frac, worst = gu.code_mismatch(q.cpu().numpy(), q_ref)
-    assert worst <= 1 and frac <= max(2 * TOL_CODES, 1.5 / q.numel() / 2)
+    assert worst <= 1 and frac <= max(TOL_CODES, 1.5 / q.numel() / 2)
 
 
 def test_glu_path_equals_plain_path_when_the_product_is_exact_in_fp16(gu):
@@ -354,9 +354,9 @@ def test_glu_path_equals_plain_path_when_the_product_is_exact_in_fp16(gu):
                 sr.quant_act(gu.dev(X), None, 0.9, q, step)
             torch.cuda.synchronize()
             outs.append((q.cpu().numpy(), step.cpu().numpy()))
-        assert np.abs(outs[0][1] / outs[1][1] - 1).max() <= 2e-6
+        assert np.abs(outs[0][1] / outs[1][1] - 1).max() <= TOL_SCALE
         frac, worst = gu.code_mismatch(outs[0][0], outs[1][0])
-        assert worst <= 1 and frac <= 1e-3
+        assert worst <= 1 and frac <= max(2 * TOL_CODES, 1.5 / outs[0][0].size / 2)   # two GPU paths, each within TOL_CODES of the oracle
 
 
 # ------------------------------------------------ weight clip-ratio search
@@ -386,7 +386,11 @@ def test_weight_clip_search_matches_oracle(gu, K, N, slices):
     rows = np.arange(N)
     # the chosen ratio minimises the oracle's error curve (up to the fp32 noise of the rotation)
     assert np.all(errs[rows, best] <= errs.min(axis=1) * (1 + 1e-4) + 1e-30)
-    assert (best != best_ref).mean() <= 0.1
+    # wherever the GPU took another ratio than the oracle, the oracle's own two errors are a tie up
+    # to the fp32 noise of the rotation: its error curve decides, not a share of rows
+    differ = best != best_ref
+    e_gpu, e_ref = errs[rows, best], errs[rows, best_ref]
+    assert np.all(np.abs(e_gpu[differ] - e_ref[differ]) <= 1e-6 * e_ref[differ] + 1e-30), (e_gpu[differ], e_ref[differ])
     assert best[2] == 0 and step[2] == np.float32(1.0) and best[3] == 0
     # staged: the oracle's quantizer at the ratio the GPU chose
     for r in rows:

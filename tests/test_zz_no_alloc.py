@@ -52,6 +52,12 @@ def test_static_scratch_entry_point_matches_linear_twice_in_a_row():
         rel = (np.abs(got - want).max(axis=1) / np.abs(want).max(axis=1)).max()
         assert rel <= TOL_OUT, (call, rel)
         assert np.array_equal(got, want)               # same kernels, same order of integer sums
+        # and directly against the CPU oracle on the same codes and steps
+        from oracle import smoothrot_oracle as orc
+        xq_h, dx_h, wq_h, dw_h = _case(100 + call, M, N, K)
+        Y_orc = orc.linear(xq_h, dx_h, wq_h, dw_h).astype(np.float64)
+        rel_orc = (np.abs(got - Y_orc).max(axis=1) / np.abs(Y_orc).max(axis=1)).max()
+        assert rel_orc <= TOL_OUT, (call, rel_orc)
 
 
 def test_static_scratch_entry_point_refuses_oversized_shapes_and_needs_no_scratch_for_prefill():
