@@ -409,7 +409,7 @@ walsh4096_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
     if (*lost != 0) break;
 #pragma unroll
     for (int g = 0; g < 8; ++g) {
-      const __half2* h = reinterpret_cast<const __half2*>(&raw[g]);
+      const uint32_t* h = reinterpret_cast<const uint32_t*>(&raw[g]);
       float4 p0, p1;
       if (kHasPre) {
         p0 = *reinterpret_cast<const float4*>(spre + g * 512 + t * 8);
@@ -417,8 +417,7 @@ walsh4096_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
       }
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
-        const float2 f = __half22float2(h[k]);
-        f32x2 val = pack2(f.x, f.y);
+        f32x2 val = half2_to_f32x2(h[k]);   // on the FMA pipe; cvt.f32.f16 would queue on the conversion unit
         if (kHasPre) {
           const f32x2 pp = k == 0 ? pack2(p0.x, p0.y) : k == 1 ? pack2(p0.z, p0.w)
                          : k == 2 ? pack2(p1.x, p1.y) : pack2(p1.z, p1.w);
@@ -464,14 +463,14 @@ walsh4096_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
     continue;
   }
 
-  float amax = 0.0f;
+  float am[4] = {0.0f, 0.0f, 0.0f, 0.0f};   // four chains: the maximum is not one long dependency
 #pragma unroll
   for (int u = 0; u < 32; ++u) {
     float a, b;
     unpack2(v[u], a, b);
-    amax = fmaxf(amax, fmaxf(fabsf(a), fabsf(b)));
+    am[u & 3] = fmaxf(fmaxf(am[u & 3], fabsf(a)), fabsf(b));
   }
-  amax = warp_max(amax);
+  float amax = warp_max(fmaxf(fmaxf(am[0], am[1]), fmaxf(am[2], am[3])));
   if (lane == 0) red[group][t >> 5] = amax;
   group_barrier(group);
   amax = fmaxf(red[group][0], red[group][1]) * 0.015625f;   // now the absmax of the normalised row
