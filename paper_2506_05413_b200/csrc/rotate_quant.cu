@@ -825,7 +825,7 @@ paley512_kernel(const __half* __restrict__ X, int64_t ldx, const __half* __restr
       }
     }
 
-    const float isk = 0.00835190877f;   // 1 / sqrt(14336), rounded to fp32
+    const float isk = 0.00835191381f;   // 1 / sqrt(14336), rounded to fp32
     if (!kQuant) {
       {
         float* y = y_out + m * kP512K + a2 * 512;
@@ -902,6 +902,10 @@ paley512_kernel(const __half* __restrict__ X, int64_t ldx, const __half* __restr
   }  // rows of this group
 }
 
+}  // namespace smoothrot
+#include "paley512_tc.cuh"
+namespace smoothrot {
+
 // ---------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------
@@ -977,6 +981,31 @@ static int launch_rotate(const void* X, int64_t rows, int64_t K, int64_t ld, con
     const int sms = device_sm_count();
     const unsigned grid = unsigned(rows < sms ? rows : sms);
     kern<<<grid, kW4096Threads, kW4096SmemBytes, stream>>>(x, ld, rows, pre, clip, q_out, step_out, y_out);
+    count_launch();
+    return launch_status();
+  }
+  if (K == kP512K && !glu && pre == nullptr && rows >= 256) {
+    // No diagonal: the Walsh part of the rotation on the tensor cores (paley512_tc.cuh).
+    const bool low = kQuant && (7.0f / clip >= 8.49f);
+    // the rows as a [rows][28][8 blocks of 64][64 values] tensor; a box = one block of 64 values of the 28 rows a
+    CUtensorMap xmap;
+    TensorMapEncodeFn encode = tensor_map_encoder();
+    if (encode == nullptr) return SMOOTHROT_CUDA_ERROR;
+    const cuuint64_t dims[4] = {64, 8, 28, cuuint64_t(rows)};
+    const cuuint64_t strides[3] = {128, 1024, cuuint64_t(ld) * sizeof(__half)};
+    const cuuint32_t box[4] = {64, 1, 28, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    if (encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<__half*>(x), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return SMOOTHROT_CUDA_ERROR;
+    auto kern = low ? ptc::paley512_tc_kernel<kQuant, true> : ptc::paley512_tc_kernel<kQuant, false>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ptc::kSmemBytes) != cudaSuccess)
+      return SMOOTHROT_CUDA_ERROR;
+    const int64_t batches = (rows + ptc::kTokens - 1) / ptc::kTokens;
+    const int sms = device_sm_count();
+    const unsigned grid = unsigned(batches < sms ? batches : sms);
+    kern<<<grid, ptc::kThreads, ptc::kSmemBytes, stream>>>(xmap, rows, clip, q_out, step_out, y_out);
     count_launch();
     return launch_status();
   }

@@ -447,3 +447,48 @@ def test_kv_quantizer_rejects_bad_arguments(gu):
     s = torch.empty((2, 1), dtype=torch.float32, device=gu.DEV)
     with pytest.raises(sr.SmoothRotError):
         sr.kv_quant(X, 0.95, q, s, s.clone())
+
+
+# ------------------------------------------------ tensor-core rotation kernels (no diagonal, many rows)
+@pytest.mark.parametrize("K,M", [(4096, 512), (4096, 777), (4096, 7200), (14336, 256), (14336, 301), (14336, 1030)])
+def test_tensor_core_rotation_and_codes_match_oracle(gu, K, M):
+    """Without a diagonal and with a few hundred rows or more, K = 4096 and K = 14336 run their Walsh
+    factor of order 128 / 256 on tcgen05: the rotation export, the steps and the codes against the
+    oracle, on rows that include massive outliers, an all-zero row, the ends of the fp16 range and a
+    single spike, with a row stride larger than K and a ragged last batch."""
+    import torch
+    from paper_2506_05413_b200 import binding as sr
+    rng = np.random.default_rng(K + M)
+    ld = K + 24
+    Xfull = np.zeros((M, ld), np.float16)
+    X = rng.standard_normal((M, K)).astype(np.float32)
+    X[::17, rng.choice(K, 3, replace=False)] *= 1500.0        # massive outliers on some tokens
+    X[1] = 0.0
+    X[2] = 65504.0
+    X[3] = -65504.0
+    X[4] = 0.0
+    X[4, K // 3] = 3.0                                        # a single spike
+    X[M - 1] *= 1e-3                                          # a small row at the ragged end
+    Xfull[:, :K] = np.clip(X, -65504, 65504).astype(np.float16)
+    Xd = gu.dev(Xfull)[:, :K]                                 # strided view
+    Xh = Xfull[:, :K]
+    # rotation alone
+    Y = torch.empty((M, K), dtype=torch.float32, device=gu.DEV)
+    sr.debug_hadamard(Xd, None, Y)
+    torch.cuda.synchronize()
+    assert sr.device_status() == 0
+    rows = np.unique(np.concatenate([np.arange(8), [M - 2, M - 1], rng.choice(M, 24, replace=False)]))
+    ref = orc.rotate(Xh[rows], None, K)
+    assert gu.rowwise_rel(Y.cpu().numpy()[rows], ref) <= TOL_ROT
+    # quantized, two clip ratios (0.8 reaches the two-sided clamp)
+    for clip in (0.9, 0.8):
+        q = torch.empty((M, K // 2), dtype=torch.uint8, device=gu.DEV)
+        step = torch.empty(M, dtype=torch.float32, device=gu.DEV)
+        sr.quant_act(Xd, None, clip, q, step)
+        torch.cuda.synchronize()
+        assert sr.device_status() == 0
+        q_ref, step_ref, _ = orc.quant_act(Xh[rows], None, K, clip)
+        assert np.abs(step.cpu().numpy()[rows] / step_ref - 1).max() <= TOL_SCALE
+        frac, worst = gu.code_mismatch(q.cpu().numpy()[rows], q_ref)
+        assert worst <= 1 and frac <= TOL_CODES, (clip, frac, worst)
+        assert step.cpu().numpy()[1] == np.float32(1.0) and not q.cpu().numpy()[1].any()
