@@ -122,6 +122,97 @@ __device__ __forceinline__ void load_half(uint32_t dst, const CUtensorMap* map, 
       : "memory");
 }
 
+// The part of the epilogue after the tensor-memory load: r[g] is the order-128 factor's output i of
+// group g of one token (position 128 g + i), unnormalised; `norm` times the final value is the
+// rotated entry (2^-6, times the inverse of a power-of-two scale the caller may have applied).
+// Order-32 factor over g in registers, row maximum over the 128 threads that share the token
+// (they meet at named barrier `barrier_id`; `mine` is their four-float exchange slot), step,
+// rounding by the 1.5 * 2^23 trick, and packing: the codes of eight consecutive positions meet
+// through warp shuffles.
+template <bool kQuant, bool kLowClamp>
+__device__ __forceinline__ void finish_token(float* r, float norm, int i, int lane, int quarter, volatile float* mine,
+                                             int barrier_id, float clip, int64_t m, uint8_t* __restrict__ q_out,
+                                             float* __restrict__ step_out, float* __restrict__ y_out) {
+  const bool odd = (i & 1) != 0;
+  const int r4 = (i >> 1) & 3;
+  const uint32_t sel1 = (r4 & 1) ? 0x3715u : 0x6240u;
+  const uint32_t sel2 = (r4 & 2) ? 0x3276u : 0x5410u;
+  // the order-32 factor over the groups g: r[g] is position 128 g + i
+  f32x2 v[16];
+#pragma unroll
+  for (int p = 0; p < 16; ++p) v[p] = pack2(r[2 * p] + r[2 * p + 1], r[2 * p] - r[2 * p + 1]);
+  butterflies_between_pairs<16>(v);
+
+  if (!kQuant) {
+    float* y = y_out + m * 4096 + i;
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      float a, c;
+      unpack2(v[p], a, c);
+      y[(2 * p) * 128] = a * norm;
+      y[(2 * p + 1) * 128] = c * norm;
+    }
+    return;
+  }
+
+  float am[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+  for (int p = 0; p < 16; ++p) {
+    float a, c;
+    unpack2(v[p], a, c);
+    am[p & 3] = fmaxf(fmaxf(am[p & 3], fabsf(a)), fabsf(c));
+  }
+  float amax = warp_max(fmaxf(fmaxf(am[0], am[1]), fmaxf(am[2], am[3])));
+  if (lane == 0) mine[quarter] = amax;
+  asm volatile("bar.sync %0, 128;" ::"r"(barrier_id) : "memory");
+  amax = fmaxf(fmaxf(mine[0], mine[1]), fmaxf(mine[2], mine[3])) * norm;
+  const float step = step_from_absmax(amax, clip);
+  if (i == 0) step_out[m] = step;
+  const float inv = __frcp_rn(step) * norm;
+  const f32x2 inv2 = pack2(inv, inv);
+  const float kMagic = 12582912.0f + 8.0f;  // 1.5 * 2^23 + 8: low byte = code + 8
+  const f32x2 magic2 = pack2(kMagic, kMagic);
+  uint32_t spread[8];                       // four codes per word, one per byte: groups 4 w .. 4 w + 3
+#pragma unroll
+  for (int w = 0; w < 8; ++w) {
+    uint32_t c4[4];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      float q0, q1;
+      unpack2(fma2(v[2 * w + k], inv2, magic2), q0, q1);
+      if (kLowClamp) {
+        q0 = fmaxf(fminf(q0, 12582912.0f + 15.0f), 12582912.0f);
+        q1 = fmaxf(fminf(q1, 12582912.0f + 15.0f), 12582912.0f);
+      }
+      c4[2 * k] = __float_as_uint(q0);
+      c4[2 * k + 1] = __float_as_uint(q1);
+    }
+    uint32_t four = __byte_perm(__byte_perm(c4[0], c4[1], 0x0040), __byte_perm(c4[2], c4[3], 0x0040), 0x5410);
+    if (!kLowClamp) four -= (four >> 4) & 0x01010101u;   // the code +8 comes down to +7
+    spread[w] = four;
+  }
+  // Lanes 2p and 2p + 1 hold the even and the odd position of each output byte: the even lane
+  // finishes the words with even w, the odd lane those with odd w.
+  uint32_t* q = reinterpret_cast<uint32_t*>(q_out + m * 2048) + (i >> 3);
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const uint32_t give = odd ? spread[2 * c] : spread[2 * c + 1];
+    const uint32_t keep = odd ? spread[2 * c + 1] : spread[2 * c];
+    const uint32_t got = __shfl_xor_sync(0xffffffffu, give, 1);
+    const uint32_t lo_n = odd ? got : keep;   // even position -> low nibble
+    const uint32_t hi_n = odd ? keep : got;
+    uint32_t wd = (lo_n | (hi_n << 4)) ^ 0x88888888u;   // offset binary -> two's complement
+    // byte k of wd: group 4 (2c + odd) + k, output byte 64 g + (i >> 1).  A 4 x 4 byte transpose
+    // among the lanes (i >> 1) & 3 = 0..3 turns these into aligned 32-bit words.
+    uint32_t pw = __shfl_xor_sync(0xffffffffu, wd, 2);
+    wd = __byte_perm(wd, pw, sel1);
+    pw = __shfl_xor_sync(0xffffffffu, wd, 4);
+    wd = __byte_perm(wd, pw, sel2);
+    const int g = 4 * (2 * c + (odd ? 1 : 0)) + r4;
+    q[g * 16] = wd;
+  }
+}
+
 template <bool kQuant, bool kLowClamp, int kTokens>
 __global__ void __launch_bounds__(Cfg<kTokens>::kThreads, 1)
 walsh4096_tc_kernel(const __grid_constant__ CUtensorMap xmap, int64_t M, float clip,
@@ -244,10 +335,6 @@ walsh4096_tc_kernel(const __grid_constant__ CUtensorMap xmap, int64_t M, float c
     const int quarter = warp & 3;            // the tensor-memory lanes this warp may read: 32 quarter .. + 31
     const int slot = (warp - 4) >> 2;        // takes the tokens slot, slot + kEpiSlots, .. of a batch
     const int i = quarter * 32 + lane;       // output index inside a group (position = 128 g + i)
-    const bool odd = (i & 1) != 0;
-    const int r4 = (i >> 1) & 3;
-    const uint32_t sel1 = (r4 & 1) ? 0x3715u : 0x6240u;
-    const uint32_t sel2 = (r4 & 2) ? 0x3276u : 0x5410u;
     uint32_t it = 0, tok_count = 0;
     bool ok = true;
     for (int64_t b = blockIdx.x; b < batches && ok; b += gridDim.x, ++it) {
@@ -262,82 +349,9 @@ walsh4096_tc_kernel(const __grid_constant__ CUtensorMap xmap, int64_t M, float c
         float r[32];
         tmem_load32(tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(ab * 256 + tk * 32), r);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        // the order-32 factor over the groups g: r[g] is position 128 g + i
-        f32x2 v[16];
-#pragma unroll
-        for (int p = 0; p < 16; ++p) v[p] = pack2(r[2 * p] + r[2 * p + 1], r[2 * p] - r[2 * p + 1]);
-        butterflies_between_pairs<16>(v);
-
-        if (!kQuant) {
-          float* y = y_out + m * 4096 + i;
-#pragma unroll
-          for (int p = 0; p < 16; ++p) {
-            float a, c;
-            unpack2(v[p], a, c);
-            y[(2 * p) * 128] = a * 0.015625f;
-            y[(2 * p + 1) * 128] = c * 0.015625f;
-          }
-          continue;
-        }
-
-        float am[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-#pragma unroll
-        for (int p = 0; p < 16; ++p) {
-          float a, c;
-          unpack2(v[p], a, c);
-          am[p & 3] = fmaxf(fmaxf(am[p & 3], fabsf(a)), fabsf(c));
-        }
-        float amax = warp_max(fmaxf(fmaxf(am[0], am[1]), fmaxf(am[2], am[3])));
-        volatile float* mine = red + (slot * 2 + (tok_count & 1)) * 4;
-        if (lane == 0) mine[quarter] = amax;
-        asm volatile("bar.sync %0, 128;" ::"r"(1 + slot) : "memory");
-        amax = fmaxf(fmaxf(mine[0], mine[1]), fmaxf(mine[2], mine[3])) * 0.015625f;
+        finish_token<kQuant, kLowClamp>(r, 0.015625f, i, lane, quarter, red + (slot * 2 + (tok_count & 1)) * 4, 1 + slot,
+                                         clip, m, q_out, step_out, y_out);
         ++tok_count;
-        const float step = step_from_absmax(amax, clip);
-        if (i == 0) step_out[m] = step;
-        const float inv = __frcp_rn(step) * 0.015625f;
-        const f32x2 inv2 = pack2(inv, inv);
-        const float kMagic = 12582912.0f + 8.0f;  // 1.5 * 2^23 + 8: low byte = code + 8
-        const f32x2 magic2 = pack2(kMagic, kMagic);
-        uint32_t spread[8];                       // four codes per word, one per byte: groups 4 w .. 4 w + 3
-#pragma unroll
-        for (int w = 0; w < 8; ++w) {
-          uint32_t c4[4];
-#pragma unroll
-          for (int k = 0; k < 2; ++k) {
-            float q0, q1;
-            unpack2(fma2(v[2 * w + k], inv2, magic2), q0, q1);
-            if (kLowClamp) {
-              q0 = fmaxf(fminf(q0, 12582912.0f + 15.0f), 12582912.0f);
-              q1 = fmaxf(fminf(q1, 12582912.0f + 15.0f), 12582912.0f);
-            }
-            c4[2 * k] = __float_as_uint(q0);
-            c4[2 * k + 1] = __float_as_uint(q1);
-          }
-          uint32_t four = __byte_perm(__byte_perm(c4[0], c4[1], 0x0040), __byte_perm(c4[2], c4[3], 0x0040), 0x5410);
-          if (!kLowClamp) four -= (four >> 4) & 0x01010101u;   // the code +8 comes down to +7
-          spread[w] = four;
-        }
-        // Lanes 2p and 2p + 1 hold the even and the odd position of each output byte: the even lane
-        // finishes the words with even w, the odd lane those with odd w.
-        uint32_t* q = reinterpret_cast<uint32_t*>(q_out + m * 2048) + (i >> 3);
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const uint32_t give = odd ? spread[2 * c] : spread[2 * c + 1];
-          const uint32_t keep = odd ? spread[2 * c + 1] : spread[2 * c];
-          const uint32_t got = __shfl_xor_sync(0xffffffffu, give, 1);
-          const uint32_t lo_n = odd ? got : keep;   // even position -> low nibble
-          const uint32_t hi_n = odd ? keep : got;
-          uint32_t wd = (lo_n | (hi_n << 4)) ^ 0x88888888u;   // offset binary -> two's complement
-          // byte k of wd: group 4 (2c + odd) + k, output byte 64 g + (i >> 1).  A 4 x 4 byte transpose
-          // among the lanes (i >> 1) & 3 = 0..3 turns these into aligned 32-bit words.
-          uint32_t pw = __shfl_xor_sync(0xffffffffu, wd, 2);
-          wd = __byte_perm(wd, pw, sel1);
-          pw = __shfl_xor_sync(0xffffffffu, wd, 4);
-          wd = __byte_perm(wd, pw, sel2);
-          const int g = 4 * (2 * c + (odd ? 1 : 0)) + r4;
-          q[g * 16] = wd;
-        }
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();

@@ -450,15 +450,28 @@ def test_kv_quantizer_rejects_bad_arguments(gu):
 
 
 # ------------------------------------------------ tensor-core rotation kernels (no diagonal, many rows)
-@pytest.mark.parametrize("K,M", [(4096, 512), (4096, 777), (4096, 7200), (14336, 256), (14336, 301), (14336, 1030)])
-def test_tensor_core_rotation_and_codes_match_oracle(gu, K, M):
+@pytest.mark.parametrize("K,M,diag", [(4096, 512, None), (4096, 777, None), (4096, 7200, None), (14336, 256, None),
+                                      (14336, 301, None), (14336, 1030, None), (4096, 1024, "smooth"),
+                                      (4096, 1101, "wide"), (4096, 6150, "smooth"), (4096, 1027, "tiny")])
+def test_tensor_core_rotation_and_codes_match_oracle(gu, K, M, diag):
     """Without a diagonal and with a few hundred rows or more, K = 4096 and K = 14336 run their Walsh
     factor of order 128 / 256 on tcgen05: the rotation export, the steps and the codes against the
-    oracle, on rows that include massive outliers, an all-zero row, the ends of the fp16 range and a
-    single spike, with a row stride larger than K and a ragged last batch."""
+    oracle, on rows that include massive outliers, an all-zero row, the ends of the fp16 range, a
+    single spike and a row a thousand times smaller than the rest, with a row stride larger than K
+    and a ragged last batch.  The same rows with diagonals (smoothing-like with a dead channel, six
+    decades wide with random signs, uniformly tiny) take the register kernel at these row counts."""
     import torch
     from paper_2506_05413_b200 import binding as sr
     rng = np.random.default_rng(K + M)
+    pre = None
+    if diag == "smooth":
+        pre = (rng.uniform(0.08, 0.3, K) * rng.choice([-1.0, 1.0], K)).astype(np.float32)
+        pre[rng.choice(K, 4, replace=False)] = 0.004          # channels that carry the outliers
+        pre[5] = 89.0                                         # a dead channel
+    elif diag == "wide":
+        pre = (10.0 ** rng.uniform(-3, 3, K) * rng.choice([-1.0, 1.0], K)).astype(np.float32)
+    elif diag == "tiny":
+        pre = (rng.uniform(1.0, 2.0, K) * 3e-7).astype(np.float32)
     ld = K + 24
     Xfull = np.zeros((M, ld), np.float16)
     X = rng.standard_normal((M, K)).astype(np.float32)
@@ -474,20 +487,21 @@ def test_tensor_core_rotation_and_codes_match_oracle(gu, K, M):
     Xh = Xfull[:, :K]
     # rotation alone
     Y = torch.empty((M, K), dtype=torch.float32, device=gu.DEV)
-    sr.debug_hadamard(Xd, None, Y)
+    pre_d = gu.dev(pre) if pre is not None else None
+    sr.debug_hadamard(Xd, pre_d, Y)
     torch.cuda.synchronize()
     assert sr.device_status() == 0
     rows = np.unique(np.concatenate([np.arange(8), [M - 2, M - 1], rng.choice(M, 24, replace=False)]))
-    ref = orc.rotate(Xh[rows], None, K)
+    ref = orc.rotate(Xh[rows], pre, K)
     assert gu.rowwise_rel(Y.cpu().numpy()[rows], ref) <= TOL_ROT
     # quantized, two clip ratios (0.8 reaches the two-sided clamp)
     for clip in (0.9, 0.8):
         q = torch.empty((M, K // 2), dtype=torch.uint8, device=gu.DEV)
         step = torch.empty(M, dtype=torch.float32, device=gu.DEV)
-        sr.quant_act(Xd, None, clip, q, step)
+        sr.quant_act(Xd, pre_d, clip, q, step)
         torch.cuda.synchronize()
         assert sr.device_status() == 0
-        q_ref, step_ref, _ = orc.quant_act(Xh[rows], None, K, clip)
+        q_ref, step_ref, _ = orc.quant_act(Xh[rows], pre, K, clip)
         assert np.abs(step.cpu().numpy()[rows] / step_ref - 1).max() <= TOL_SCALE
         frac, worst = gu.code_mismatch(q.cpu().numpy()[rows], q_ref)
         assert worst <= 1 and frac <= TOL_CODES, (clip, frac, worst)
