@@ -373,8 +373,11 @@ walsh4096_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
                                                          kW4096Groups * 8) + group;
 
   if (kHasPre) {
+    // the diagonal's 16-byte unit i = (g, t, half) goes to (g, half, t): the two units a thread reads
+    // per chunk are then 1 KB apart and the lanes of a warp read consecutive units (no bank conflicts)
     for (int i = threadIdx.x; i < 1024; i += kW4096Threads)
-      reinterpret_cast<float4*>(spre)[i] = __ldg(reinterpret_cast<const float4*>(pre) + i);
+      reinterpret_cast<float4*>(spre)[(i & ~127) | ((i & 1) << 6) | ((i >> 1) & 63)] =
+          __ldg(reinterpret_cast<const float4*>(pre) + i);
   }
   if (t == 0) {
     *lost = 0;
@@ -412,8 +415,8 @@ walsh4096_kernel(const __half* __restrict__ X, int64_t ldx, int64_t M,
       const uint32_t* h = reinterpret_cast<const uint32_t*>(&raw[g]);
       float4 p0, p1;
       if (kHasPre) {
-        p0 = *reinterpret_cast<const float4*>(spre + g * 512 + t * 8);
-        p1 = *reinterpret_cast<const float4*>(spre + g * 512 + t * 8 + 4);
+        p0 = reinterpret_cast<const float4*>(spre)[g * 128 + t];
+        p1 = reinterpret_cast<const float4*>(spre)[g * 128 + 64 + t];
       }
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
