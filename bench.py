@@ -97,6 +97,21 @@ def profiled_traffic(M, N, K):
     return None
 
 
+def profiled_traffic_of(label):
+    """Same, for a kernel that is not the GEMM: a line `dram_bytes_per_launch <label>: <bytes>`."""
+    pat = re.compile(r"dram_bytes_per_launch\s+" + re.escape(label) + r":\s*([0-9.eE+]+)")
+    folder = os.path.join(ROOT, "profiles")
+    if not os.path.isdir(folder):
+        return None
+    for name in sorted(os.listdir(folder)):
+        if name.endswith((".md", ".txt")):
+            with open(os.path.join(folder, name)) as f:
+                m = pat.search(f.read())
+                if m:
+                    return float(m.group(1))
+    return None
+
+
 def layer_ops(M, N, K):
     return 2.0 * M * N * K
 
@@ -701,6 +716,20 @@ def run_gpu(args, case, desc):
                 "Lambda^-1 absorbed by the producing layer); timed alone, not part of the step"}
     per_call["clocks"] = clocks_calls
 
+    # the memory-bound kernel of the online path, against the copy bandwidth
+    def hbm_roofline(kernel, seconds, label):
+        got = abytes["quant_act"] / seconds / 1e9
+        return {"kernel": kernel, "bound": "hbm", "achieved": got, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": got / peaks["hbm_gbs"], "traffic": profiled_traffic_of(label),
+                "algorithmic_bytes": abytes["quant_act"],
+                "timed": "CUDA events around back-to-back launches of this call alone, inputs rotated out of L2",
+                "peak_source": f"{peaks['source']} copy bandwidth"}
+    roofline_quant = {
+        "diagonal": hbm_roofline("smoothrot_quant_act, diagonal d/s (register kernel)", call_ms["quant_act"] * 1e-3,
+                                 f"quant_act rows={M} K={K} diagonal=1"),
+        "no_diagonal": hbm_roofline("smoothrot_quant_act, no diagonal", exact_mean,
+                                    f"quant_act rows={M} K={K} diagonal=0")}
+
     # ---- the other workloads, one GPU only (each with its own clock record) ----
     per_config = None
     if args.per_config and world == 1:
@@ -739,6 +768,7 @@ def run_gpu(args, case, desc):
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
         "gpu_launches": int(launches),
         "roofline": roofline,
+        "roofline_quant_act": roofline_quant,
         "peaks": rec,
         "cpu_baseline": {"value": cpu_value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
                          "sample": sample},

@@ -114,7 +114,7 @@ int smoothrot_fuse_weights_search(const void* W_f16, int64_t N, int64_t K, int64
   if (!aligned16(workspace)) return SMOOTHROT_BAD_ALIGNMENT;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   auto kern = clip_search_kernel;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(row_bytes)) != cudaSuccess)
+  if (!allow_dynamic_smem(reinterpret_cast<const void*>(kern), int(row_bytes)))
     return SMOOTHROT_CUDA_ERROR;
   const int64_t slice = int64_t(workspace_bytes / row_bytes) < N ? int64_t(workspace_bytes / row_bytes) : N;
   const __half* W = static_cast<const __half*>(W_f16);

@@ -6,6 +6,8 @@
 #include <stdint.h>
 
 #include <atomic>
+#include <mutex>
+#include <vector>
 
 #include "smoothrot.h"
 
@@ -78,6 +80,29 @@ inline TensorMapEncodeFn tensor_map_encoder() {
   return fn;
 }
 #endif
+
+// Raises a kernel's dynamic shared-memory limit: one runtime call per kernel, device and size, then a
+// table look-up (the runtime call costs a microsecond or so on every eager launch otherwise).
+inline bool allow_dynamic_smem(const void* kern, int bytes) {
+  struct Entry {
+    const void* kern;
+    int dev;
+    int bytes;
+  };
+  static std::mutex mu;
+  static std::vector<Entry> done;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    for (const Entry& e : done)
+      if (e.kern == kern && e.dev == dev && e.bytes >= bytes) return true;
+  }
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+  std::lock_guard<std::mutex> lock(mu);
+  done.push_back(Entry{kern, dev, bytes});
+  return true;
+}
 
 inline int launch_status() {
   return cudaGetLastError() == cudaSuccess ? SMOOTHROT_OK : SMOOTHROT_CUDA_ERROR;

@@ -962,12 +962,12 @@ static int launch_rotate(const void* X, int64_t rows, int64_t K, int64_t ld, con
     const unsigned grid = unsigned(batches < sms ? batches : sms);
     if (six) {
       auto kern = low ? wtc::walsh4096_tc_kernel<kQuant, true, 6> : wtc::walsh4096_tc_kernel<kQuant, false, 6>;
-      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, wtc::Cfg<6>::kSmemBytes) != cudaSuccess)
+      if (!allow_dynamic_smem(reinterpret_cast<const void*>(kern), wtc::Cfg<6>::kSmemBytes))
         return SMOOTHROT_CUDA_ERROR;
       kern<<<grid, wtc::Cfg<6>::kThreads, wtc::Cfg<6>::kSmemBytes, stream>>>(xmap, rows, clip, q_out, step_out, y_out);
     } else {
       auto kern = low ? wtc::walsh4096_tc_kernel<kQuant, true, 4> : wtc::walsh4096_tc_kernel<kQuant, false, 4>;
-      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, wtc::Cfg<4>::kSmemBytes) != cudaSuccess)
+      if (!allow_dynamic_smem(reinterpret_cast<const void*>(kern), wtc::Cfg<4>::kSmemBytes))
         return SMOOTHROT_CUDA_ERROR;
       kern<<<grid, wtc::Cfg<4>::kThreads, wtc::Cfg<4>::kSmemBytes, stream>>>(xmap, rows, clip, q_out, step_out, y_out);
     }
@@ -979,7 +979,7 @@ static int launch_rotate(const void* X, int64_t rows, int64_t K, int64_t ld, con
     const bool low = kQuant && (7.0f / clip >= 8.49f);
     auto kern = pre ? (low ? walsh4096_kernel<kQuant, true, true> : walsh4096_kernel<kQuant, true, false>)
                     : (low ? walsh4096_kernel<kQuant, false, true> : walsh4096_kernel<kQuant, false, false>);
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kW4096SmemBytes) != cudaSuccess)
+    if (!allow_dynamic_smem(reinterpret_cast<const void*>(kern), kW4096SmemBytes))
       return SMOOTHROT_CUDA_ERROR;
     const int sms = device_sm_count();
     const unsigned grid = unsigned(rows < sms ? rows : sms);
@@ -1003,7 +1003,7 @@ static int launch_rotate(const void* X, int64_t rows, int64_t K, int64_t ld, con
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return SMOOTHROT_CUDA_ERROR;
     auto kern = low ? ptc::paley512_tc_kernel<kQuant, true> : ptc::paley512_tc_kernel<kQuant, false>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ptc::kSmemBytes) != cudaSuccess)
+    if (!allow_dynamic_smem(reinterpret_cast<const void*>(kern), ptc::kSmemBytes))
       return SMOOTHROT_CUDA_ERROR;
     const int64_t batches = (rows + ptc::kTokens - 1) / ptc::kTokens;
     const int sms = device_sm_count();
@@ -1020,7 +1020,7 @@ static int launch_rotate(const void* X, int64_t rows, int64_t K, int64_t ld, con
                  : (low ? paley512_kernel<kQuant, false, true, kG> : paley512_kernel<kQuant, false, false, kG>);
     };
     auto kern = glu ? pick(std::true_type{}) : pick(std::false_type{});
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kP512SmemBytes) != cudaSuccess)
+    if (!allow_dynamic_smem(reinterpret_cast<const void*>(kern), kP512SmemBytes))
       return SMOOTHROT_CUDA_ERROR;
     const int sms = device_sm_count();
     const unsigned grid = unsigned(rows < sms ? rows : sms);
@@ -1030,7 +1030,7 @@ static int launch_rotate(const void* X, int64_t rows, int64_t K, int64_t ld, con
   }
   const size_t smem = size_t(K) * sizeof(float);
   auto kern = glu ? rotate_generic_kernel<kQuant, true> : rotate_generic_kernel<kQuant, false>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
+  if (!allow_dynamic_smem(reinterpret_cast<const void*>(kern), int(smem)))
     return SMOOTHROT_CUDA_ERROR;
   const float inv_sqrt_k = float(1.0 / sqrt(double(K)));
   kern<<<unsigned(rows), kGenericThreads, smem, stream>>>(x, ld, u, ldu, int(K), base, n, logn, pre, inv_sqrt_k, clip,

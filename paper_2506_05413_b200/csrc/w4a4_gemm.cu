@@ -1583,30 +1583,66 @@ static EncodeTiledFn encode_fn() {
   return fn;
 }
 
+// A tensor map is a pure function of (address, shape, box); the last few are kept so that repeated
+// eager calls on the same buffers (a layer called once per step) do not encode them again.
+template <typename Build>
+static bool cached_map(CUtensorMap* map, int kind, const void* ptr, int64_t d0, int64_t d1, int64_t d2, Build build) {
+  struct Entry {
+    int kind;
+    const void* ptr;
+    int64_t d0, d1, d2;
+    CUtensorMap map;
+  };
+  constexpr int kEntries = 16;
+  static std::mutex mu;
+  static Entry table[kEntries];
+  static int filled = 0, next = 0;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    for (int i = 0; i < filled; ++i) {
+      const Entry& e = table[i];
+      if (e.kind == kind && e.ptr == ptr && e.d0 == d0 && e.d1 == d1 && e.d2 == d2) {
+        *map = e.map;
+        return true;
+      }
+    }
+  }
+  if (!build(map)) return false;
+  std::lock_guard<std::mutex> lock(mu);
+  table[next] = Entry{kind, ptr, d0, d1, d2, *map};
+  next = (next + 1) % kEntries;
+  if (filled < kEntries) ++filled;
+  return true;
+}
+
 // 2-D map over a packed matrix [rows x K/2] bytes, box = 64 bytes x box_rows, 64-byte swizzle.
 static bool make_map(CUtensorMap* map, const uint8_t* ptr, int64_t rows, int64_t K, int box_rows) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
-  const cuuint64_t dims[2] = {cuuint64_t(K / 2), cuuint64_t(rows)};
-  const cuuint64_t strides[1] = {cuuint64_t(K / 2)};
-  const cuuint32_t box[2] = {cuuint32_t(kPackedRow), cuuint32_t(box_rows)};
-  const cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(ptr), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return cached_map(map, 0, ptr, rows, K, box_rows, [&](CUtensorMap* out) {
+    const cuuint64_t dims[2] = {cuuint64_t(K / 2), cuuint64_t(rows)};
+    const cuuint64_t strides[1] = {cuuint64_t(K / 2)};
+    const cuuint32_t box[2] = {cuuint32_t(kPackedRow), cuuint32_t(box_rows)};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  });
 }
 
 // 2-D map over the fp16 output [M x ldy], box = 64 columns x 32 rows, 128-byte swizzle (TMA stores).
 static bool make_map_y(CUtensorMap* map, __half* Y, int64_t M, int64_t N, int64_t ldy) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
-  const cuuint64_t dims[2] = {cuuint64_t(N), cuuint64_t(M)};
-  const cuuint64_t strides[1] = {cuuint64_t(ldy) * sizeof(__half)};
-  const cuuint32_t box[2] = {64, 32};
-  const cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, Y, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
-         CUDA_SUCCESS;
+  return cached_map(map, 1, Y, M, N, ldy, [&](CUtensorMap* out) {
+    const cuuint64_t dims[2] = {cuuint64_t(N), cuuint64_t(M)};
+    const cuuint64_t strides[1] = {cuuint64_t(ldy) * sizeof(__half)};
+    const cuuint32_t box[2] = {64, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, Y, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+           CUDA_SUCCESS;
+  });
 }
 
 // Raises a kernel's dynamic shared-memory limit; once per kernel, device and process.  kTag tells
