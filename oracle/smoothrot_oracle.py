@@ -130,25 +130,60 @@ def paley28() -> np.ndarray:
     return (np.eye(q + 1, dtype=np.int64) + S).astype(np.int8)
 
 
+def legendre(e: int, q: int) -> int:
+    """Quadratic character of the prime field GF(q): 0 at zero, +1 on the non-zero squares
+    y*y mod q, -1 otherwise (the squares are found by listing them)."""
+    e %= q
+    if e == 0:
+        return 0
+    return 1 if any((y * y) % q == e for y in range(1, q)) else -1
+
+
+def paley_prime(q: int) -> np.ndarray:
+    """Paley construction I for a prime q = 3 mod 4, same conventions as paley28 with the
+    field elements 0..q-1 in their natural order: Q[a, b] = chi(a - b), S = [[0, 1^T], [-1, Q]],
+    H = I + S of order q + 1.  An addition for layer widths 12 * 2^p and 20 * 2^p (q = 11, 19);
+    the paper's models need the orders 2^p and 28 * 2^p only."""
+    assert q in (11, 19), "only the orders 12 and 20 are built this way"
+    S = np.zeros((q + 1, q + 1), dtype=np.int64)
+    S[0, 1:] = 1
+    S[1:, 0] = -1
+    for a in range(q):
+        for b in range(q):
+            S[1 + a, 1 + b] = legendre(a - b, q)
+    return (np.eye(q + 1, dtype=np.int64) + S).astype(np.int8)
+
+
+def base_matrix(base: int) -> np.ndarray:
+    """The small factor of the Kronecker product: Paley I of order 12, 20 or 28."""
+    if base == 28:
+        return paley28()
+    if base in (12, 20):
+        return paley_prime(base - 1)
+    raise ValueError(f"no base matrix of order {base}")
+
+
 def split_order(K: int):
-    """K = base * 2^p with base 1 (Walsh) or 28 (Paley x Walsh).  Returns (base, 2^p)."""
+    """K = base * 2^p with base 1 (Walsh) or 4 * odd for odd in {3, 5, 7}: 12, 20, 28 (Paley x Walsh).
+    The odd part of K decides the base, so the split is unique.  Returns (base, 2^p)."""
     if K >= 1 and (K & (K - 1)) == 0:
         return 1, K
-    if K % 28 == 0:
-        n = K // 28
-        if n >= 1 and (n & (n - 1)) == 0:
-            return 28, n
+    for base in (28, 20, 12):
+        if K >= base and K % base == 0:
+            n = K // base
+            if (n & (n - 1)) == 0:
+                return base, n
     raise ValueError(f"no Hadamard construction for order {K}")
 
 
 def hadamard_matrix(K: int) -> np.ndarray:
     """The +1/-1 matrix H of order K used for the rotation: Sylvester for 2^p,
-    and for 28 * 2^p the Kronecker product with the Paley matrix on the slow
-    index:  H[a*n + b, a'*n + b'] = H28[a, a'] * Hn[b, b']."""
+    and for base * 2^p the Kronecker product with the Paley matrix on the slow
+    index:  H[a*n + b, a'*n + b'] = Hbase[a, a'] * Hn[b, b']."""
     base, n = split_order(K)
     if base == 1:
         return sylvester(n)
-    return np.kron(paley28().astype(np.int8), sylvester(n)).astype(np.int8)
+    return np.kron(base_matrix(base).astype(np.int8), sylvester(n)).astype(np.int8)
 
 
 # ---------------------------------------------------------------------------
@@ -181,9 +216,9 @@ def _walsh_last_axis(v: np.ndarray) -> np.ndarray:
 
 
 def rotate(x: np.ndarray, pre, K: int) -> np.ndarray:
-    """Same map as rotate_dense, by float64 butterflies: for K = 28 * n the row
-    is viewed as [28, n], the Walsh transform runs along n and the Paley
-    matrix along the 28-axis (the Kronecker product, factor by factor)."""
+    """Same map as rotate_dense, by float64 butterflies: for K = base * n the row
+    is viewed as [base, n], the Walsh transform runs along n and the Paley
+    matrix along the base axis (the Kronecker product, factor by factor)."""
     v = np.asarray(x, dtype=np.float64)
     assert v.ndim == 2 and v.shape[1] == K
     if pre is not None:
@@ -193,8 +228,8 @@ def rotate(x: np.ndarray, pre, K: int) -> np.ndarray:
         y = _walsh_last_axis(v)
     else:
         w = _walsh_last_axis(v.reshape(v.shape[0], base, n))
-        P = paley28().astype(np.float64)
-        # y[m, a', b] = sum_a w[m, a, b] * H28[a, a']
+        P = base_matrix(base).astype(np.float64)
+        # y[m, a', b] = sum_a w[m, a, b] * Hbase[a, a']
         y = np.einsum("mab,ac->mcb", w, P).reshape(v.shape[0], K)
     return y / np.sqrt(np.float64(K))
 

@@ -123,19 +123,61 @@ def test_order_14336_rows_are_orthogonal():
     assert np.array_equal(G, want)
     A = orc.paley28().astype(np.int64)
     B = orc.sylvester(512).astype(np.int64)
-    assert np.array_equal(np.kron(A @ A.T, B @ B.T), K * np.eye(K, dtype=np.int64))
+    # (A x B)(A x B)^T = (A A^T) x (B B^T) = (28 I) x (512 I) = 14336 I
+    assert np.array_equal(A @ A.T, 28 * np.eye(28, dtype=np.int64))
+    assert np.array_equal(B @ B.T, 512 * np.eye(512, dtype=np.int64))
 
 
 def test_split_order():
     assert orc.split_order(4096) == (1, 4096)
     assert orc.split_order(14336) == (28, 512)
     assert orc.split_order(28) == (28, 1)
-    for bad in (0, 3, 12, 11008, 28 * 3):
+    assert orc.split_order(12) == (12, 1)
+    assert orc.split_order(5120) == (20, 256)
+    assert orc.split_order(3072) == (12, 256)
+    for bad in (0, 3, 11008, 28 * 3, 36, 60, 44):
         with pytest.raises(ValueError):
             orc.split_order(bad)
 
 
-@pytest.mark.parametrize("K", [128, 512, 28 * 4, 28 * 16, 1024])
+@pytest.mark.parametrize("q", [11, 19])
+def test_paley_prime_structure(q):
+    """Orders 12 and 20: the same structure facts as for order 28, and the character checked
+    against Euler's criterion e^((q-1)/2) mod q (another route to it than listing squares)."""
+    n = q + 1
+    H = orc.paley_prime(q).astype(np.int64)
+    assert H.shape == (n, n) and set(np.unique(H)) == {-1, 1}
+    assert np.array_equal(H @ H.T, n * np.eye(n, dtype=np.int64))
+    assert np.array_equal(H.T @ H, n * np.eye(n, dtype=np.int64))
+    S = H - np.eye(n, dtype=np.int64)
+    assert np.array_equal(S, -S.T)
+    Q = S[1:, 1:]
+    assert np.all(np.diag(Q) == 0) and np.all(Q.sum(axis=1) == 0) and np.all(Q.sum(axis=0) == 0)
+    assert np.array_equal(Q @ Q.T, q * np.eye(q, dtype=np.int64) - np.ones((q, q), np.int64))
+    assert np.all(H[0] == 1) and np.all(H[1:, 0] == -1)
+    for e in range(q):
+        euler = pow(e, (q - 1) // 2, q)
+        assert orc.legendre(e, q) == {0: 0, 1: 1, q - 1: -1}[euler]
+    for a in range(q):                      # circulant: Q[a, b] = chi(a - b)
+        for b in range(q):
+            assert Q[a, b] == Q[(a - b) % q, 0]
+    assert orc.legendre(-1, q) == -1        # q = 3 mod 4: -1 is a non-square, Q is skew
+
+
+@pytest.mark.parametrize("K", [12 * 8, 20 * 16])
+def test_kronecker_with_orders_12_and_20(K):
+    base, n = orc.split_order(K)
+    H = orc.hadamard_matrix(K).astype(np.int64)
+    assert np.array_equal(H @ H.T, K * np.eye(K, dtype=np.int64))
+    P, Wn = orc.base_matrix(base).astype(int), orc.sylvester(n).astype(int)
+    rng = np.random.default_rng(K)
+    for _ in range(16):
+        a, a2 = rng.integers(base, size=2)
+        b, b2 = rng.integers(n, size=2)
+        assert H[a * n + b, a2 * n + b2] == P[a, a2] * Wn[b, b2]
+
+
+@pytest.mark.parametrize("K", [128, 512, 28 * 4, 28 * 16, 1024, 12 * 32, 20 * 8])
 def test_fast_rotation_equals_dense_definition(K):
     rng = np.random.default_rng(K)
     x = rng.standard_normal((5, K))
@@ -159,7 +201,7 @@ def test_fast_rotation_equals_dense_on_full_width_rows(K):
     assert np.abs(got - want).max() <= 1e-12 * np.abs(want).max()
 
 
-@pytest.mark.parametrize("K", [128, 4096, 28 * 32, 14336])
+@pytest.mark.parametrize("K", [128, 4096, 28 * 32, 14336, 3072, 5120])
 def test_rotation_closed_forms(K):
     rng = np.random.default_rng(K + 1)
     base, n = orc.split_order(K)
