@@ -12,6 +12,9 @@
  *                     K = 2^p : Sylvester / Walsh, H[i][j] = (-1)^popcount(i & j)
  *                     K = 28 * 2^p : kron(H28, H_{2^p}), index j = a * 2^p + b,
  *                     H28 = Paley construction I over GF(27) (smoothrot_paley28)
+ *                     K = 12 * 2^p, 20 * 2^p : the same with Paley I over GF(11), GF(19)
+ *                     (smoothrot_base_matrix; an addition for other layer widths, the
+ *                     paper's models need only the two forms above)
  *
  * The equivalent transformation (Eq. 2 of the paper) is
  *   Y = (X diag(pre_x) H / sqrt(K)) (W diag(pre_w) H / sqrt(K))^T,
@@ -33,7 +36,7 @@
  *   - Leading dimensions (ldx, ldw, ldy) count elements, not bytes.
  *   - fp16 inputs must be 16-byte aligned with leading dimensions that are
  *     multiples of 8; packed tensors must be 16-byte aligned.
- *   - K must be 2^p with 7 <= p <= 13, or 28 * 2^p with 3 <= p <= 9.
+ *   - K must be 2^p with 7 <= p <= 13, or 12 * 2^p, 20 * 2^p or 28 * 2^p with 3 <= p <= 10.
  *   - Return value: SMOOTHROT_OK (0) or a negative smoothrot_status.  On an
  *     error nothing has been enqueued.  A size of zero rows is valid and
  *     enqueues nothing.
@@ -327,6 +330,11 @@ int smoothrot_debug_wait_expiry(void* stream);
 /* Host. Writes the library's own order-28 Paley matrix, row-major, entries
  * +1 / -1, into out[784] (a host buffer). */
 int smoothrot_paley28(int8_t* out_host);
+
+/* Host. The same for the small factor of order 12, 20 or 28 (Paley construction I over GF(11),
+ * GF(19), GF(27); first row all +1, first column +1 then -1): order * order entries, row-major,
+ * into a host buffer.  SMOOTHROT_INVALID_ARG for another order or a null pointer. */
+int smoothrot_base_matrix(int order, int8_t* out_host);
 
 /*
  * Host, synchronous.  Kernels never spin without bound: a wait that runs out

@@ -43,6 +43,7 @@ SIGNATURES = {
     "smoothrot_debug_set_wait_limit_ns": (_int, [ctypes.c_uint64]),
     "smoothrot_debug_wait_expiry": (_int, [_vp]),
     "smoothrot_paley28": (_int, [_vp]),
+    "smoothrot_base_matrix": (_int, [_int, _vp]),
     "smoothrot_device_status": (_int, [ctypes.POINTER(_int), _int]),
     "smoothrot_launch_count": (_i64, []),
 }
@@ -353,6 +354,14 @@ def paley28():
     buf = (ctypes.c_int8 * 784)()
     _check(load().smoothrot_paley28(ctypes.cast(buf, ctypes.c_void_p)))
     return [[int(buf[r * 28 + c]) for c in range(28)] for r in range(28)]
+
+
+def base_matrix(order: int):
+    """The library's Paley matrix of order 12, 20 or 28 as a list of rows of +1/-1 (host call)."""
+    order = int(order)
+    buf = (ctypes.c_int8 * (order * order))()
+    _check(load().smoothrot_base_matrix(order, ctypes.cast(buf, ctypes.c_void_p)))
+    return [[int(buf[r * order + c]) for c in range(order)] for r in range(order)]
 
 
 def debug_set_wait_limit_ns(ns: int) -> None:

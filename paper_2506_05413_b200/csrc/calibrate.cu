@@ -167,7 +167,7 @@ const char* smoothrot_status_string(int status) {
   switch (status) {
     case SMOOTHROT_OK: return "ok";
     case SMOOTHROT_INVALID_ARG: return "invalid argument";
-    case SMOOTHROT_UNSUPPORTED_K: return "unsupported K (need 2^p, 7<=p<=13, or 28*2^p, 3<=p<=9)";
+    case SMOOTHROT_UNSUPPORTED_K: return "unsupported K (need 2^p, 7<=p<=13, or 12*2^p, 20*2^p, 28*2^p, 3<=p<=10)";
     case SMOOTHROT_BAD_ALIGNMENT: return "pointer or leading dimension not aligned";
     case SMOOTHROT_WORKSPACE_TOO_SMALL: return "workspace too small";
     case SMOOTHROT_CUDA_ERROR: return "CUDA error";

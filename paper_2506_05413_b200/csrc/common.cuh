@@ -28,8 +28,8 @@ inline int ilog2(int64_t v) {
   return l;
 }
 
-// K = base * n with base 1 (Walsh, n = 2^p, 7 <= p <= 13) or base 28
-// (Paley x Walsh, n = 2^p, 3 <= p <= 9).  Returns false if K is neither.
+// K = base * n with base 1 (Walsh, n = 2^p, 7 <= p <= 13) or base 12, 20 or 28
+// (Paley x Walsh, n = 2^p, 3 <= p <= 10).  Returns false if K is neither.
 inline bool split_order(int64_t K, int* base, int* n, int* logn) {
   if (is_pow2(K)) {
     int l = ilog2(K);
@@ -37,11 +37,14 @@ inline bool split_order(int64_t K, int* base, int* n, int* logn) {
     *base = 1; *n = int(K); *logn = l;
     return true;
   }
-  if (K > 0 && K % 28 == 0 && is_pow2(K / 28)) {
-    int l = ilog2(K / 28);
-    if (l < 3 || l > 9) return false;
-    *base = 28; *n = int(K / 28); *logn = l;
-    return true;
+  // 4 * odd * 2^p with odd in {3, 5, 7}: the odd part of K decides the Paley factor (12, 20 or 28)
+  for (int b : {28, 20, 12}) {
+    if (K > 0 && K % b == 0 && is_pow2(K / b)) {
+      int l = ilog2(K / b);
+      if (l < 3 || l > 10) return false;
+      *base = b; *n = int(K / b); *logn = l;
+      return true;
+    }
   }
   return false;
 }

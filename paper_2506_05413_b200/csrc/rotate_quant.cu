@@ -8,7 +8,7 @@
 // Kernels
 //   rotate_generic_kernel   any supported K; one CTA per row, the row lives in
 //                           shared memory as fp32, butterflies three bits at a
-//                           time, the order-28 factor by a table product.
+//                           time, the order-12, -20 or -28 factor by a table product.
 //   walsh4096_kernel        K = 4096: 64 threads per row, 64 values per thread,
 //                           6 + 6 butterfly stages in registers around one
 //                           shared-memory transpose, codes assembled with warp
@@ -78,6 +78,40 @@ constexpr Paley28Table make_paley28_table() {
 
 __constant__ Paley28Table c_paley28 = make_paley28_table();
 
+// Orders 12 and 20: Paley construction I over the prime fields GF(11) and GF(19), elements
+// 0..q-1 in natural order, same border as above.  (Widths 12 * 2^p and 20 * 2^p; an addition,
+// the paper's models need 2^p and 28 * 2^p only.)
+__host__ __device__ constexpr int prime_character(int e, int q) {
+  e = ((e % q) + q) % q;
+  if (e == 0) return 0;
+  int acc = 1;                                 // Euler's criterion: e^((q-1)/2) mod q
+  for (int i = 0; i < (q - 1) / 2; ++i) acc = (acc * e) % q;
+  return acc == 1 ? 1 : -1;
+}
+
+__host__ __device__ constexpr int paley_prime_entry(int q, int r, int c) {
+  if (r == 0) return 1;
+  if (c == 0) return -1;
+  if (r == c) return 1;
+  return prime_character((r - 1) - (c - 1), q);
+}
+
+template <int kOrder>
+struct PaleyTable {
+  float v[kOrder][kOrder];
+};
+
+template <int kOrder>
+constexpr PaleyTable<kOrder> make_paley_prime_table() {
+  PaleyTable<kOrder> t{};
+  for (int r = 0; r < kOrder; ++r)
+    for (int c = 0; c < kOrder; ++c) t.v[r][c] = float(paley_prime_entry(kOrder - 1, r, c));
+  return t;
+}
+
+__constant__ PaleyTable<12> c_paley12 = make_paley_prime_table<12>();
+__constant__ PaleyTable<20> c_paley20 = make_paley_prime_table<20>();
+
 // ---------------------------------------------------------------------------
 // Small device helpers
 // ---------------------------------------------------------------------------
@@ -101,6 +135,25 @@ __device__ __forceinline__ float glu_product(float g, float u) {
 // Generic kernel: one CTA per row.
 // ---------------------------------------------------------------------------
 constexpr int kGenericThreads = 256;
+
+template <int kOrder>
+__device__ __forceinline__ void base_product(float* row, const float (&table)[kOrder][kOrder], int n, int tid) {
+  for (int b = tid; b < n; b += kGenericThreads) {
+    float xin[kOrder], yv[kOrder];
+#pragma unroll
+    for (int a = 0; a < kOrder; ++a) xin[a] = row[a * n + b];
+#pragma unroll
+    for (int c = 0; c < kOrder; ++c) {
+      float acc = 0.0f;
+#pragma unroll
+      for (int a = 0; a < kOrder; ++a) acc = fmaf(xin[a], table[a][c], acc);
+      yv[c] = acc;
+    }
+#pragma unroll
+    for (int c = 0; c < kOrder; ++c) row[c * n + b] = yv[c];
+  }
+  __syncthreads();
+}
 
 template <bool kQuant, bool kGlu>
 __global__ void __launch_bounds__(kGenericThreads)
@@ -167,24 +220,10 @@ rotate_generic_kernel(const __half* __restrict__ X, int64_t ldx, const __half* _
     __syncthreads();
   }
 
-  // Order-28 factor on the slow index a of j = a * n + b:  y[a'] = sum_a x[a] H28[a][a'].
-  if (base == 28) {
-    for (int b = tid; b < n; b += kGenericThreads) {
-      float xin[28], yv[28];
-#pragma unroll
-      for (int a = 0; a < 28; ++a) xin[a] = row[a * n + b];
-#pragma unroll
-      for (int c = 0; c < 28; ++c) {
-        float acc = 0.0f;
-#pragma unroll
-        for (int a = 0; a < 28; ++a) acc = fmaf(xin[a], c_paley28.v[a][c], acc);
-        yv[c] = acc;
-      }
-#pragma unroll
-      for (int c = 0; c < 28; ++c) row[c * n + b] = yv[c];
-    }
-    __syncthreads();
-  }
+  // Paley factor on the slow index a of j = a * n + b:  y[a'] = sum_a x[a] H[a][a'].
+  if (base == 28) base_product<28>(row, c_paley28.v, n, tid);
+  else if (base == 20) base_product<20>(row, c_paley20.v, n, tid);
+  else if (base == 12) base_product<12>(row, c_paley12.v, n, tid);
 
   if (!kQuant) {
     float* y = y_out + m * int64_t(K);
@@ -1094,6 +1133,15 @@ int smoothrot_rotate_status_word(int* value, int clear) {
 int smoothrot_rotate_set_wait_limit_ns(uint64_t ns) {
   const unsigned long long v = ns == 0 ? smoothrot::kLoadWaitLimitNs : static_cast<unsigned long long>(ns);
   if (cudaMemcpyToSymbol(smoothrot::g_rotate_wait_limit_ns, &v, sizeof(v)) != cudaSuccess) return SMOOTHROT_CUDA_ERROR;
+  return SMOOTHROT_OK;
+}
+
+int smoothrot_base_matrix(int order, int8_t* out_host) {
+  if (out_host == nullptr || (order != 12 && order != 20 && order != 28)) return SMOOTHROT_INVALID_ARG;
+  for (int r = 0; r < order; ++r)
+    for (int c = 0; c < order; ++c)
+      out_host[r * order + c] = int8_t(order == 28 ? smoothrot::paley28_entry(r, c)
+                                                   : smoothrot::paley_prime_entry(order - 1, r, c));
   return SMOOTHROT_OK;
 }
 

@@ -46,7 +46,7 @@ def test_host_side_rejections(lib):
     q = lib.smoothrot_quant_act
     assert q(dummy, 4, 100, 104, None, 0.9, dummy, dummy, None) == -2        # unsupported K
     assert q(dummy, 4, 64, 64, None, 0.9, dummy, dummy, None) == -2          # 2^6 too small
-    assert q(dummy, 4, 28 * 1024, 28 * 1024, None, 0.9, dummy, dummy, None) == -2
+    assert q(dummy, 4, 28 * 2048, 28 * 2048, None, 0.9, dummy, dummy, None) == -2
     assert q(dummy, -1, 128, 128, None, 0.9, dummy, dummy, None) == -1       # negative rows
     assert q(None, 4, 128, 128, None, 0.9, dummy, dummy, None) == -1         # null input
     assert q(dummy, 4, 128, 64, None, 0.9, dummy, dummy, None) == -1         # ld < K
@@ -55,7 +55,7 @@ def test_host_side_rejections(lib):
     assert q(dummy, 4, 128, 128, None, 0.0, dummy, dummy, None) == -1        # clip out of range
     assert q(dummy, 4, 128, 128, None, 1.5, dummy, dummy, None) == -1
     assert q(dummy, 0, 128, 128, None, 0.9, None, None, None) == 0           # empty input is fine
-    assert lib.smoothrot_fuse_weights(dummy, 4, 96, 96, None, 1.0, dummy, dummy, None) == -2
+    assert lib.smoothrot_fuse_weights(dummy, 4, 88, 88, None, 1.0, dummy, dummy, None) == -2
     qp = lib.smoothrot_quant_act_plain
     assert qp(dummy, 4, 100, 104, None, 0.9, dummy, dummy, None) == -2           # K % 8
     assert qp(dummy, 4, 32768, 32768, None, 0.9, dummy, dummy, None) == -2       # K too long
@@ -102,6 +102,7 @@ def test_host_side_rejections(lib):
     assert cal(dummy, 4, 128, 128, dummy, 4, 128, 1.5, 1, dummy, dummy, None, None, None, None) == -1  # alpha
     assert cal(dummy, 4, 128, 128, None, 0, 0, 0.5, 0, None, None, None, None, None, None) == -1
     assert lib.smoothrot_paley28(None) == -1
+    assert lib.smoothrot_base_matrix(12, None) == -1
     assert lib.smoothrot_device_status(None, 0) == -1
 
 
@@ -110,3 +111,6 @@ def test_library_paley_table_equals_oracle_table(lib):
     from oracle import smoothrot_oracle as orc
     from paper_2506_05413_b200 import binding
     assert np.array_equal(np.array(binding.paley28(), dtype=np.int8), orc.paley28())
+    for order in (12, 20, 28):
+        assert np.array_equal(np.array(binding.base_matrix(order), dtype=np.int8), orc.base_matrix(order))
+    assert lib.smoothrot_base_matrix(16, None) == -1

@@ -45,7 +45,8 @@ def _pre(seed, K):
 
 # ------------------------------------------------------------------ rotation
 @pytest.mark.parametrize("K,M", [(128, 64), (256, 5), (512, 33), (1024, 7), (2048, 3), (4096, 37),
-                                 (4096, 4), (8192, 2), (28 * 8, 9), (28 * 64, 5), (14336, 11)])
+                                 (4096, 4), (8192, 2), (28 * 8, 9), (28 * 64, 5), (14336, 11),
+                                 (12 * 8, 6), (12 * 256, 5), (20 * 16, 9), (20 * 256, 4), (28 * 1024, 2)])
 @pytest.mark.parametrize("use_pre", [False, True])
 def test_rotation_matches_oracle(gu, K, M, use_pre):
     X = _acts(K + M, M, K)
@@ -81,7 +82,8 @@ def test_rotation_with_row_stride(gu):
 
 
 # ------------------------------------------------------- quantize + pack
-@pytest.mark.parametrize("K,M", [(128, 64), (512, 21), (4096, 301), (4096, 1), (8192, 3), (28 * 16, 10), (14336, 19)])
+@pytest.mark.parametrize("K,M", [(128, 64), (512, 21), (4096, 301), (4096, 1), (8192, 3), (28 * 16, 10), (14336, 19),
+                                 (12 * 256, 17), (20 * 256, 13), (28 * 1024, 3)])
 @pytest.mark.parametrize("which", ["act", "weight"])
 def test_quantized_codes_match_oracle(gu, K, M, which):
     from paper_2506_05413_b200 import binding as sr
