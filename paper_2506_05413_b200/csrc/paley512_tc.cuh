@@ -128,11 +128,19 @@ paley512_tc_kernel(const __grid_constant__ CUtensorMap xmap, int64_t M, float cl
                     4 * (kb >> 1) + 2 * c + (kb & 1), int(b * kTokens + tk));
   };
 
+  // The first batch's copy goes out before anything else (it needs one barrier only and has the
+  // longest latency of the set-up); the second stage is requested after the set-up barrier.
   uint32_t produced = 0;
   if (threadIdx.x == 0) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(&xmap) : "memory");
+    wtc::mbar_init(full(0), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (int64_t(blockIdx.x) < batches) {
+      issue_batch(0, int64_t(blockIdx.x));
+      produced = 1;
+    }
     for (int s = 0; s < kStages; ++s) {
-      wtc::mbar_init(full(s), 1);
+      if (s > 0) wtc::mbar_init(full(s), 1);
       wtc::mbar_init(empty(s), 1);
     }
     for (int s = 0; s < 2; ++s) {
@@ -141,8 +149,6 @@ paley512_tc_kernel(const __grid_constant__ CUtensorMap xmap, int64_t M, float cl
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    for (int64_t b = blockIdx.x; b < batches && produced < uint32_t(kStages); b += gridDim.x, ++produced)
-      issue_batch(int(produced), b);
   }
   // H128 and -H128 in the operand's form: row i = 128 bytes per K half, 16-byte unit u at u ^ (i & 7).
   // The slots 28..31 of every (c, token) are never written by TMA: zero them once (their columns
