@@ -452,7 +452,7 @@ def test_kv_quantizer_rejects_bad_arguments(gu):
 
 
 # ------------------------------------------------ tensor-core rotation kernels (no diagonal, many rows)
-@pytest.mark.parametrize("K,M,diag", [(4096, 512, None), (4096, 777, None), (4096, 7200, None), (14336, 256, None),
+@pytest.mark.parametrize("K,M,diag", [(4096, 512, None), (4096, 777, None), (4096, 7200, None), (4096, 7992, None), (14336, 256, None),
                                       (14336, 301, None), (14336, 1030, None), (4096, 1024, "smooth"),
                                       (4096, 1101, "wide"), (4096, 6150, "smooth"), (4096, 1027, "tiny")])
 def test_tensor_core_rotation_and_codes_match_oracle(gu, K, M, diag):
