@@ -186,6 +186,7 @@ GEMM_SHAPES = [
     (70, 1000, 1024),    # 2 k-splits added up inside a cluster, ragged channels
     (80, 520, 4096),     # 8 k-splits in a cluster
     (128, 1024, 4096),
+    (128, 6144, 4096),   # 48 channel tiles: 2 k-splits keep the CTAs in one wave
     (100, 256, 16384),   # few channels, long K: k-splits through the workspace
     (128, 256, 8192),
     (300, 1024, 2048),   # 3 token tiles of the streaming kernel, ragged
