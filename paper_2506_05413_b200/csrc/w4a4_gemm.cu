@@ -1513,6 +1513,79 @@ static int sm_count() {
 
 constexpr int kPairSplitMinBlocks = 32;   // k-blocks per split below which the extra pass over the partial sums costs more than it saves
 
+// Clusters of `size` CTAs of the streaming kernel that the device runs at the same time.  A cluster
+// stays inside one GPC, so large clusters leave SMs unused: 148 / 74 / 33 / 15 clusters of
+// 1 / 2 / 4 / 8 on B200.  Asked of the runtime once per device; a conservative guess without one.
+static int active_clusters(int size) {
+  constexpr int kSlots = 64;
+  static std::atomic<int> cached[kSlots][4];
+  const int idx = size >= 8 ? 3 : size >= 4 ? 2 : size >= 2 ? 1 : 0;
+  const int guess = size <= 1 ? sm_count() : sm_count() / size * 7 / 8;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kSlots) return guess;
+  int n = cached[dev][idx].load(std::memory_order_relaxed);
+  if (n > 0) return n;
+  auto kern = w4a4_gemm_stream_kernel<128>;
+  n = 0;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Stream<128>::kSmemBytes) == cudaSuccess) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(unsigned(size * 32), 1, 1);
+    cfg.blockDim = dim3(unsigned(Stream<128>::kThreads), 1, 1);
+    cfg.dynamicSmemBytes = size_t(Stream<128>::kSmemBytes);
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = unsigned(size);
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) n = 0;
+  }
+  if (n <= 0) {
+    (void)cudaGetLastError();
+    return guess;
+  }
+  cached[dev][idx].store(n, std::memory_order_relaxed);
+  return n;
+}
+
+// How the streaming kernel would split K for this shape.
+struct StreamPlan {
+  int splits;
+  bool cluster;
+  int ctas;
+};
+
+static StreamPlan plan_stream(int64_t M, int64_t N, int kblocks) {
+  const int tiles = int((N + kBM - 1) / kBM) * int((M + 127) / 128);
+  const int slots = sm_count();   // one CTA of the streaming kernel per SM
+  // as many k-splits as keep all CTAs in one wave (a second wave costs a second fill and drain:
+  // 128 tokens x 6144 channels took 24 us with 4 splits in two waves, 17 us with 2 splits in one)
+  int want = slots / tiles;
+  if (want < 1) want = 1;
+  // Workspace path: the largest divisor of kblocks that does not exceed `want` and leaves >= 4
+  // k-blocks per split.  Cluster path: the same among 1, 2, 4, 8 (portable cluster sizes that
+  // divide the 128 channels of a tile), as long as the device runs that many clusters at once.
+  // The cluster path needs no workspace and no second kernel, so it is taken unless the workspace
+  // path offers at least four times the CTAs while the cluster path would leave more than half
+  // of the machine idle.
+  int splits = 1, csplits = 1;
+  for (int s = 1; s <= kblocks && s <= want; ++s)
+    if (kblocks % s == 0 && kblocks / s >= 4) splits = s;
+  for (int s = 2; s <= 8 && s <= want; s *= 2)
+    if (kblocks % s == 0 && kblocks / s >= 4 && tiles <= active_clusters(s)) csplits = s;
+  StreamPlan sp{};
+  if (splits >= 4 * csplits && 2 * csplits * tiles < slots) {
+    sp.cluster = false;
+    sp.splits = splits;
+  } else {
+    sp.cluster = csplits > 1;
+    sp.splits = csplits;
+  }
+  sp.ctas = tiles * sp.splits;
+  return sp;
+}
+
 static Plan make_plan(int64_t M, int64_t N, int64_t K) {
   Plan pl{};
   const int kblocks = int(K / kWideRow);
@@ -1523,49 +1596,38 @@ static Plan make_plan(int64_t M, int64_t N, int64_t K) {
     pl.splits = 1;
     return pl;
   }
-  // The two-CTA kernel works on 256 x 256 tiles, one per SM pair.  Up to 256 tokens (one row of
-  // tiles) it is taken when the output channels alone fill more than half of the pairs, and the
-  // streaming kernel with 128-token tiles and k-splits otherwise; up to 512 tokens the streaming
-  // kernel still wins when the tiles are very few.
+  // The two-CTA kernel works on 256 x 256 tiles, one per SM pair; with few tiles and a long K two
+  // k-splits per tile put twice as many pairs to work (partial sums through the workspace).
   const int64_t pair_tiles = ((M + 255) / 256) * ((N + 255) / 256);
-  const bool to_stream = M <= 256 ? !(N >= 256 && 4 * pair_tiles > sm_count())
-                                  : (M <= 512 && 16 * pair_tiles <= sm_count());
+  const int pairs = sm_count() / 2;
+  const int pair_splits =
+      (2 * pair_tiles <= pairs && kblocks % 2 == 0 && kblocks / 2 >= kPairSplitMinBlocks) ? 2 : 1;
+  const StreamPlan sp = plan_stream(M, N, kblocks);
+  bool to_stream;
+  if (N < 256) {
+    // no pair tiles: the streaming kernel up to 512 tokens, the one-CTA kernel beyond
+    to_stream = M <= 512;
+  } else {
+    // Between the two, the estimated time decides (microseconds, fitted to graph-replay timings of
+    // 72 shapes with 96..768 tokens on B200: a fixed part and a cost per k-block and wave).
+    const int64_t pair_waves = (pair_tiles * pair_splits + pairs - 1) / pairs;
+    const double pair_us = 10.2 + 0.35 * double(kblocks / pair_splits) * double(pair_waves) + (pair_splits > 1 ? 5.8 : 0.0);
+    const int64_t stream_waves = (sp.ctas + sm_count() - 1) / sm_count();
+    const double stream_us = (sp.cluster ? 10.7 : (sp.splits > 1 ? 16.7 : 15.6)) +
+                             0.32 * double(kblocks / sp.splits) * double(stream_waves);
+    to_stream = stream_us < pair_us;
+  }
   if (!to_stream) {
     pl.swapped = false;
     pl.pair = N >= 256;
     pl.bn = N > 64 ? 128 : 64;   // of the one-CTA kernel that serves N < 256
-    pl.splits = 1;
-    // Few tiles and a long K: two k-splits per tile put twice as many SM pairs to work; the partial
-    // sums take the workspace path.
-    if (pl.pair && 2 * pair_tiles <= sm_count() / 2 && kblocks % 2 == 0 && kblocks / 2 >= kPairSplitMinBlocks)
-      pl.splits = 2;
+    pl.splits = pl.pair ? pair_splits : 1;
     return pl;
   }
   pl.swapped = true;
   pl.bn = 128;   // narrower token tiles were slower than this one on every shape they served
-  const int tiles = int((N + kBM - 1) / kBM) * int((M + pl.bn - 1) / pl.bn);
-  const int slots = sm_count();   // one CTA of the streaming kernel per SM
-  // as many k-splits as keep all CTAs in one wave (a second wave costs a second fill and drain:
-  // 128 tokens x 6144 channels took 24 us with 4 splits in two waves, 17 us with 2 splits in one)
-  int want = slots / tiles;
-  if (want < 1) want = 1;
-  // Workspace path: the largest divisor of kblocks that does not exceed `want` and leaves >= 4
-  // k-blocks per split.  Cluster path: the same among 1, 2, 4, 8 (portable cluster sizes that
-  // divide the 128 channels of a tile).  The cluster path needs no workspace and no second
-  // kernel, so it is taken unless the workspace path offers at least four times the CTAs while
-  // the cluster path would leave more than half of the machine idle.
-  int splits = 1, csplits = 1;
-  for (int s = 1; s <= kblocks && s <= want; ++s)
-    if (kblocks % s == 0 && kblocks / s >= 4) splits = s;
-  for (int s = 1; s <= 8 && s <= want; s *= 2)
-    if (kblocks % s == 0 && kblocks / s >= 4) csplits = s;
-  if (splits >= 4 * csplits && 2 * csplits * tiles < slots) {
-    pl.cluster = false;
-  } else {
-    pl.cluster = csplits > 1;
-    splits = csplits;
-  }
-  pl.splits = splits;
+  pl.cluster = sp.cluster;
+  pl.splits = sp.splits;
   return pl;
 }
 

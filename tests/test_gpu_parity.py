@@ -203,7 +203,8 @@ GEMM_SHAPES = [
     (100, 12296, 512),   # fewer than 256 tokens, but enough channels to fill the SM pairs
     (200, 10240, 256),
     (600, 776, 512),     # ragged in both directions
-    (300, 2560, 8192),   # two k-splits through the workspace
+    (257, 3200, 8192),   # two k-splits through the workspace
+    (300, 2560, 8192),   # few enough 128-token tiles for the streaming kernel with 2 k-splits in a cluster
     (520, 2568, 8192),   # ... ragged in both directions
 ]
 
@@ -232,7 +233,7 @@ def test_gemm_extreme_codes(gu):
                                    (300, 520, 640), (1024, 768, 4096), (16, 1000, 2048), (128, 520, 1024),
                                    (100, 256, 16384), (4, 1000, 14336), (1, 4096, 4096), (6, 1024, 4096), (16, 520, 14336),
                                    (30, 8200, 1024), (64, 520, 4096), (64, 8200, 4096), (96, 12288, 1024), (160, 520, 2048),
-                                   (12, 4104, 2048), (32, 1024, 4096), (300, 2568, 8192)])
+                                   (12, 4104, 2048), (32, 1024, 4096), (300, 2568, 8192), (520, 2568, 8192)])
 def test_linear_output_matches_oracle_on_gpu_codes(gu, M, N, K):
     rng = np.random.default_rng(M + N + K)
     xq = orc.pack_codes(synth.random_codes(M, M, K))
@@ -250,7 +251,7 @@ def test_prefill_k_split_is_optional_and_changes_nothing(gu):
     it the call runs unsplit and, the sums being integers, returns the same fp16 outputs."""
     import torch
     from paper_2506_05413_b200 import binding as sr
-    M, N, K = 300, 2568, 8192
+    M, N, K = 520, 2568, 8192
     assert sr.workspace_bytes(M, N, K) > 0
     rng = np.random.default_rng(5)
     xq = gu.dev(orc.pack_codes(synth.random_codes(1, M, K)))
