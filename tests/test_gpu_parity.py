@@ -194,9 +194,12 @@ GEMM_SHAPES = [
     (512, 1024, 14336),  # long K
     (130, 136, 640),     # two token tiles, ragged both ways
     (200, 1000, 2048),
-    # one CTA per SM, both operands through shared memory (more than 256 tokens, fewer than 256 channels)
-    (300, 136, 640),     # BN = 128
-    (257, 8, 128),       # BN = 64
+    (300, 136, 640),     # few channels, 3 token tiles
+    (257, 8, 128),
+    # one CTA per SM, both operands through shared memory (more than 512 tokens, fewer than 256 channels)
+    (600, 136, 640),     # BN = 128
+    (520, 8, 128),       # BN = 64
+    (1030, 200, 1024),
     # the two-CTA kernel
     (256, 256, 128),     # one pair tile
     (300, 520, 1152),    # several tiles and a ragged tail
