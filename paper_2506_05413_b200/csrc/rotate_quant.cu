@@ -260,7 +260,7 @@ rotate_generic_kernel(const __half* __restrict__ X, int64_t ldx, const __half* _
 }
 
 // ---------------------------------------------------------------------------
-// K = 4096.  Persistent kernel: one CTA per SM, kW4096Groups (12) row groups of
+// K = 4096.  Persistent kernel: one CTA per SM, kW4096Groups (10) row groups of
 // 64 threads (two warps) each; a group walks over rows  m, m + stride, ...
 //
 // The next row of a group is fetched by a bulk asynchronous copy
@@ -981,7 +981,7 @@ static int launch_rotate(const void* X, int64_t rows, int64_t K, int64_t ld, con
     // No diagonal: the order-128 factor of the rotation on the tensor cores (walsh4096_tc.cuh).
     // A few hundred rows or fewer finish sooner in the register kernel below (shorter set-up).
     const bool low = kQuant && (7.0f / clip >= 8.49f);
-    // the rows as a [rows][32 groups][2 halves][64 values] tensor; a box = one K half of 8 rows
+    // the rows as a [rows][32 groups][2 halves][64 values] tensor; a box = one K half of a batch's rows
     CUtensorMap xmap;
     TensorMapEncodeFn encode = tensor_map_encoder();
     if (encode == nullptr) return SMOOTHROT_CUDA_ERROR;
