@@ -925,6 +925,11 @@ w4a4_gemm_pair_tmem_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
     if (lane == 0) tma_store_wait_all();
   }
 
+  // A CTA that gave up tells its peer, which would otherwise wait for its own limit (the peer is
+  // still resident: it cannot pass the cluster barrier below before this CTA arrives there).
+  if (*abort_flag != 0)
+    asm volatile("st.shared::cluster.u32 [%0], %1;"
+                 ::"r"(map_to_cta(smem_u32(const_cast<const int*>(abort_flag)), rank ^ 1u)), "r"(1u) : "memory");
   drain_after_abort(abort_flag);
   tcgen05_fence_before();
   __syncthreads();
