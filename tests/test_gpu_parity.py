@@ -316,6 +316,15 @@ def test_reduced_configs_whole_layer(gu, maker, M, N):
     _check_layer(gu, case, _layer_on_gpu(gu, case))
 
 
+@pytest.mark.parametrize("K", [3072, 5120])
+def test_whole_layer_on_other_widths(gu, K):
+    """Widths 12 * 256 and 20 * 256 (Paley factors of order 12 and 20): the whole path, staged
+    against the oracle like the named configurations."""
+    case = synth.make_layer(f"width_{K}", seed=100 + K, M=70, K=K, N=264, T=96, law="normal",
+                            w_std=0.02, n_outlier_channels=3, outlier_gain=800.0)
+    _check_layer(gu, case, _layer_on_gpu(gu, case))
+
+
 # ------------------------------------------------ gated-linear-unit input path
 @pytest.mark.parametrize("K,M", [(128, 9), (512, 21), (4096, 5), (28 * 16, 10), (14336, 1), (14336, 37)])
 @pytest.mark.parametrize("use_pre", [False, True])
