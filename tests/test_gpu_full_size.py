@@ -173,11 +173,12 @@ def test_token_sweep_decode_shapes_in_full(env, shape):
 
 @pytest.mark.parametrize("shape,M", [("q_o", 512), ("q_o", 2048), ("q_o", 8192), ("k_v", 512), ("k_v", 2048),
                                      ("k_v", 8192), ("gate_up", 512), ("gate_up", 2048), ("gate_up", 8192),
-                                     ("down", 512), ("down", 2048)])
+                                     ("down", 512), ("down", 2048),
+                                     ("q_o", 256), ("k_v", 256), ("k_v", 768), ("down", 256)])
 def test_token_sweep_prefill_shapes_sampled(env, shape, M):
     """configs[4] at the prefill end of the sweep: every linear shape of the block at M = 512, 2048 and
-    8192 tokens (the streaming kernel with k-splits, the two-CTA kernel with and without its split-K
-    reduction), checked like the full-size workloads: calibration in full, sampled whole rows of both
+    8192 tokens, and points at 256 and 768 tokens where the kernel choice changes (the streaming
+    kernel with k-splits, the two-CTA kernel with and without its split-K reduction), checked like the full-size workloads: calibration in full, sampled whole rows of both
     quantizers, 64 whole rows and 64 whole columns of the accumulators and of the output."""
     torch, sr = env
     _check_full_size(torch, sr, synth.config4(shape, M), seed=400 + M + len(shape))
